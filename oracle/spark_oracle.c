@@ -1,0 +1,336 @@
+/*
+ * SparK oracle -- TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+ *
+ * A plain, slow CPU statement of what the SparK hot path computes, written from
+ * the paper's definitions.  It shares no code, header, table or constant with
+ * the CUDA library.  Only the tests, the smoke check and the benchmark's
+ * cpu_baseline / reference arm may call it.
+ *
+ * All sums are taken in double; stored tensors (fp32 or bf16) are widened
+ * exactly.  The one place that is deliberately NOT double is the saliency
+ * product (one IEEE round-to-nearest fp32 multiply), because a floating-point
+ * value decides an integer there (which channels are kept) and both sides must
+ * take that decision in the same precision.
+ *
+ * Passages followed (section / equation of the paper):
+ *   window mean query ......... Sec. "SparK", q-bar_i^j = (1/W) sum_t q_{i,t}^j
+ *   saliency .................. Sec. "Problem Formulation", w^j = ||q^j||_2 ||k^j||_2
+ *   top-T selection ........... Eq. (cal) and the Top_T rule below it
+ *   mask, pruned key matrix ... Sec. "Saliency Measurement and Unstructured Pruning"
+ *   mu_pruned (mu, sigma) ..... App. "Caching Pruned Channel Statistics"
+ *   recovery .................. Sec. "Channel Recovery", k~ = w~ / ||q-bar^j||_2,
+ *                               degenerate distribution w~ = mu_pruned
+ *   attention ................. Sec. "Preliminaries", softmax(q K^T / sqrt(D)) V
+ *
+ * Readings taken where the paper is silent (each listed in the design notes):
+ *   - ||q-bar^j||_2 of a scalar channel is |q-bar^j|; under GQA the G*W window
+ *     queries that share a KV head are pooled into one mean;
+ *   - recovered entries are the literal non-negative quotient mu_t / |q-bar^j|;
+ *   - |q-bar^j| is floored at qnorm_eps before dividing;
+ *   - statistics are per token, over that token's pruned channels;
+ *   - on equal saliency the lower channel index is kept;
+ *   - the 1/sqrt(D) factor scales the whole reconstructed dot product.
+ *
+ * Eviction (observation-window attention-score top-k with max pooling) is not
+ * defined by the paper, which only cites the base method and its settings
+ * (App. "Implementation": window 32, pooling kernel 7); the rule coded here is
+ * the benchmark's.  PARITY UNPINNED against the paper for oracle_evict; it is
+ * pinned only by its own invariants.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+
+static inline double load_elem(const void *base, int64_t idx, int dtype)
+{
+    if (dtype == ORACLE_F32)
+        return (double)((const float *)base)[idx];
+    uint32_t bits = (uint32_t)((const uint16_t *)base)[idx] << 16;   /* bf16 -> f32, exact */
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+int oracle_version(void) { return 1; }
+
+int oracle_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------------------------
+ * Window mean query and recovery divisor.
+ *   qbar[b][h][j] = (1/(G W)) sum_{g<G} sum_{w<W} Q_win[b][h G + g][w][j]   (double, g outer)
+ *   a[b][h][j]    = max(|qbar|, eps)
+ * q_win: [B][Hq][W][D].  qbar, a: [B][Hkv][D] float (qbar may be NULL).
+ * --------------------------------------------------------------------------------- */
+int oracle_window_mean(const void *q_win, int dtype, int B, int Hq, int Hkv, int W, int D,
+                       float eps, float *qbar, float *a)
+{
+    if (!q_win || !a || Hkv <= 0 || Hq % Hkv) return 1;
+    const int G = Hq / Hkv;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h)
+            for (int j = 0; j < D; ++j) {
+                double acc = 0.0;
+                for (int g = 0; g < G; ++g)
+                    for (int w = 0; w < W; ++w)
+                        acc += load_elem(q_win, (((int64_t)b * Hq + (h * G + g)) * W + w) * D + j, dtype);
+                float m = (float)(acc / (double)(G * W));
+                int64_t o = ((int64_t)b * Hkv + h) * D + j;
+                if (qbar) qbar[o] = m;
+                float am = fabsf(m);
+                a[o] = am > eps ? am : eps;
+            }
+    return 0;
+}
+
+typedef struct { float w; int j; } sal_t;
+
+static int sal_cmp(const void *x, const void *y)
+{
+    const sal_t *p = (const sal_t *)x, *q = (const sal_t *)y;
+    if (p->w > q->w) return -1;          /* larger saliency first */
+    if (p->w < q->w) return 1;
+    return p->j - q->j;                  /* equal saliency: lower channel first */
+}
+
+/* ---------------------------------------------------------------------------------
+ * Per-token channel pruning of the keys.
+ *   w[t][j]  = a[j] * |K[t][j]|               one fp32 multiply
+ *   kept_t   = first T channels of (w descending, j ascending)
+ *   mask[t]  bit (j % 32) of word (j / 32) set  <=>  j kept
+ *   mu[t]    = mean of w over the pruned channels (0 when T == D)
+ *   mu_all, sigma_all (optional) = mean / population std of w over all D channels
+ * k: element (b,h,t,j) at b*stride_b + h*stride_h + t*stride_t + j.
+ * mask: [B][Hkv][S_max][MW], MW = ceil(D/32).  mu: [B][Hkv][S_max].
+ * kept_idx (optional): [B][Hkv][S_max][T], ascending channel order.
+ * saliency (optional): [B][Hkv][S_max][D].
+ * Rows t >= seq_lens[b] are written as zeros.
+ * --------------------------------------------------------------------------------- */
+int oracle_compress(const void *k, int dtype, int B, int Hkv, int D,
+                    int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                    const int32_t *seq_lens, int S_max, int T, const float *a,
+                    uint32_t *mask, float *mu, int32_t *kept_idx, float *saliency,
+                    float *mu_all, float *sigma_all)
+{
+    if (!k || !seq_lens || !a || !mask || !mu || T < 1 || T > D) return 1;
+    const int MW = (D + 31) / 32;
+    int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h) {
+            sal_t *row = (sal_t *)malloc(sizeof(sal_t) * (size_t)D);
+            unsigned char *keep = (unsigned char *)malloc((size_t)D);
+            if (!row || !keep) { err = 2; free(row); free(keep); continue; }
+            const float *au = a + ((int64_t)b * Hkv + h) * D;
+            for (int t = 0; t < S_max; ++t) {
+                int64_t u = ((int64_t)b * Hkv + h) * S_max + t;
+                memset(mask + u * MW, 0, sizeof(uint32_t) * (size_t)MW);
+                mu[u] = 0.f;
+                if (mu_all) mu_all[u] = 0.f;
+                if (sigma_all) sigma_all[u] = 0.f;
+                if (kept_idx) memset(kept_idx + u * T, 0, sizeof(int32_t) * (size_t)T);
+                if (saliency) memset(saliency + u * D, 0, sizeof(float) * (size_t)D);
+                if (t >= seq_lens[b]) continue;
+                const int64_t kb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                for (int j = 0; j < D; ++j) {
+                    float kf = (float)load_elem(k, kb + j, dtype);
+                    float wj = au[j] * fabsf(kf);
+                    row[j].w = wj;
+                    row[j].j = j;
+                    if (saliency) saliency[u * D + j] = wj;
+                }
+                if (mu_all || sigma_all) {
+                    double s1 = 0.0;
+                    for (int j = 0; j < D; ++j) s1 += (double)row[j].w;
+                    double m = s1 / (double)D, s2 = 0.0;
+                    for (int j = 0; j < D; ++j) { double d = (double)row[j].w - m; s2 += d * d; }
+                    if (mu_all) mu_all[u] = (float)m;
+                    if (sigma_all) sigma_all[u] = (float)sqrt(s2 / (double)D);
+                }
+                qsort(row, (size_t)D, sizeof(sal_t), sal_cmp);
+                memset(keep, 0, (size_t)D);
+                for (int r = 0; r < T; ++r) keep[row[r].j] = 1;
+                double pruned_sum = 0.0;
+                for (int r = T; r < D; ++r) pruned_sum += (double)row[r].w;
+                mu[u] = (T < D) ? (float)(pruned_sum / (double)(D - T)) : 0.f;
+                int slot = 0;
+                for (int j = 0; j < D; ++j)
+                    if (keep[j]) {
+                        mask[u * MW + j / 32] |= (uint32_t)1 << (j % 32);
+                        if (kept_idx) kept_idx[u * T + slot] = j;
+                        ++slot;
+                    }
+            }
+            free(row);
+            free(keep);
+        }
+    return err;
+}
+
+/* ---------------------------------------------------------------------------------
+ * Decode attention with on-the-fly recovery of the pruned key entries.
+ *   path 0:  K~[t][j] = K[t][j] if kept else mu[t] / a[j];
+ *            s[t] = scale * sum_j q[j] K~[t][j]
+ *   path 1:  s[t] = scale * ( sum_{kept} q[j] K[t][j] + mu[t] * sum_{pruned} q[j]/a[j] )
+ *   p = softmax_t(s),  out[c] = sum_t p[t] V[t][c],  lse = max + ln sum exp(s - max)
+ * q: [B][Hq][D]; k, v strided as in oracle_compress; lens[b] tokens attended.
+ * scale <= 0 selects 1/sqrt(D).  out: [B][Hq][D]; lse (optional): [B][Hq];
+ * scores (optional): [B][Hq][S_max] double.  A sequence of length 0 yields zeros / -inf.
+ * --------------------------------------------------------------------------------- */
+int oracle_decode_attn(const void *q, const void *k, const void *v, int dtype,
+                       int B, int Hq, int Hkv, int D,
+                       int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                       const int32_t *lens, int S_max,
+                       const uint32_t *mask, const float *mu, const float *a,
+                       double scale, int path, float *out, float *lse, double *scores)
+{
+    if (!q || !k || !v || !lens || !mask || !mu || !a || !out || Hkv <= 0 || Hq % Hkv) return 1;
+    const int G = Hq / Hkv, MW = (D + 31) / 32;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)D);
+    int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < Hq; ++i) {
+            const int h = i / G, S = lens[b];
+            float *o = out + ((int64_t)b * Hq + i) * D;
+            for (int c = 0; c < D; ++c) o[c] = 0.f;
+            if (lse) lse[(int64_t)b * Hq + i] = -INFINITY;
+            if (S <= 0) continue;
+            double *s = (double *)malloc(sizeof(double) * (size_t)S);
+            double *kt = (double *)malloc(sizeof(double) * (size_t)D);
+            double *acc = (double *)calloc((size_t)D, sizeof(double));
+            if (!s || !kt || !acc) { err = 2; free(s); free(kt); free(acc); continue; }
+            const float *au = a + ((int64_t)b * Hkv + h) * D;
+            const int64_t qb = ((int64_t)b * Hq + i) * D;
+            for (int t = 0; t < S; ++t) {
+                const int64_t u = ((int64_t)b * Hkv + h) * S_max + t;
+                const int64_t kb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                const uint32_t *m = mask + u * MW;
+                double dot = 0.0;
+                if (path == 0) {
+                    for (int j = 0; j < D; ++j) {
+                        int kept = (m[j / 32] >> (j % 32)) & 1u;
+                        kt[j] = kept ? load_elem(k, kb + j, dtype) : (double)mu[u] / (double)au[j];
+                    }
+                    for (int j = 0; j < D; ++j) dot += load_elem(q, qb + j, dtype) * kt[j];
+                } else {
+                    double kept_dot = 0.0, r = 0.0;
+                    for (int j = 0; j < D; ++j) {
+                        int kept = (m[j / 32] >> (j % 32)) & 1u;
+                        double qj = load_elem(q, qb + j, dtype);
+                        if (kept) kept_dot += qj * load_elem(k, kb + j, dtype);
+                        else r += qj / (double)au[j];
+                    }
+                    dot = kept_dot + (double)mu[u] * r;
+                }
+                s[t] = scale * dot;
+                if (scores) scores[((int64_t)b * Hq + i) * S_max + t] = s[t];
+            }
+            double mx = s[0];
+            for (int t = 1; t < S; ++t) if (s[t] > mx) mx = s[t];
+            double den = 0.0;
+            for (int t = 0; t < S; ++t) den += exp(s[t] - mx);
+            for (int t = 0; t < S; ++t) {
+                const double p = exp(s[t] - mx) / den;
+                const int64_t vb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                for (int c = 0; c < D; ++c) acc[c] += p * load_elem(v, vb + c, dtype);
+            }
+            for (int c = 0; c < D; ++c) o[c] = (float)acc[c];
+            if (lse) lse[(int64_t)b * Hq + i] = (float)(mx + log(den));
+            free(s); free(kt); free(acc);
+        }
+    return err;
+}
+
+/* ---------------------------------------------------------------------------------
+ * Eviction pre-step (benchmark rule; see the header: parity unpinned).
+ *   A_i[w][t] = softmax over t <= S-W+w of  Q_win[i][w] . K[h][t] / sqrt(D)
+ *   vote[t]   = sum_{i in group} sum_w A_i[w][t]              for t < S-W
+ *   pooled[t] = max_{|u-t| <= (pool-1)/2, 0 <= u < S-W} vote[u]
+ *   keep the (budget - W) prefix tokens of largest pooled (ties: lower t) plus the
+ *   W window tokens, in original order.  budget >= S keeps everything.
+ * kept_tok: [B][Hkv][budget] int32 (entries past out_len are -1); out_len: [B].
+ * vote_out / pooled_out (optional): [B][Hkv][S_max] double.
+ * --------------------------------------------------------------------------------- */
+typedef struct { double p; int t; } tok_t;
+
+static int tok_cmp(const void *x, const void *y)
+{
+    const tok_t *a = (const tok_t *)x, *b = (const tok_t *)y;
+    if (a->p > b->p) return -1;
+    if (a->p < b->p) return 1;
+    return a->t - b->t;
+}
+
+int oracle_evict(const void *q_win, const void *k, int dtype, int B, int Hq, int Hkv, int W, int D,
+                 int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                 const int32_t *seq_lens, int S_max, int budget, int pool,
+                 int32_t *kept_tok, int32_t *out_len, double *vote_out, double *pooled_out)
+{
+    if (!q_win || !k || !seq_lens || !kept_tok || !out_len || Hkv <= 0 || Hq % Hkv) return 1;
+    if (budget < W || pool < 1 || !(pool & 1)) return 1;
+    const int G = Hq / Hkv, half = (pool - 1) / 2;
+    const double scale = 1.0 / sqrt((double)D);
+    int err = 0;
+    for (int b = 0; b < B; ++b) {
+        const int S = seq_lens[b];
+        out_len[b] = S < budget ? S : budget;
+    }
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h) {
+            const int S = seq_lens[b];
+            int32_t *kt = kept_tok + ((int64_t)b * Hkv + h) * budget;
+            for (int r = 0; r < budget; ++r) kt[r] = -1;
+            if (S <= budget) { for (int t = 0; t < S; ++t) kt[t] = t; continue; }
+            if (S < W) { err = 3; continue; }
+            const int P = S - W;                         /* prefix length */
+            double *vote = (double *)calloc((size_t)S, sizeof(double));
+            double *s = (double *)malloc(sizeof(double) * (size_t)S);
+            tok_t *cand = (tok_t *)malloc(sizeof(tok_t) * (size_t)P);
+            unsigned char *sel = (unsigned char *)calloc((size_t)S, 1);
+            if (!vote || !s || !cand || !sel) { err = 2; free(vote); free(s); free(cand); free(sel); continue; }
+            for (int g = 0; g < G; ++g)
+                for (int w = 0; w < W; ++w) {
+                    const int i = h * G + g, last = P + w;          /* causal: attends t <= last */
+                    const int64_t qb = (((int64_t)b * Hq + i) * W + w) * D;
+                    double mx = -INFINITY;
+                    for (int t = 0; t <= last; ++t) {
+                        const int64_t kb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                        double dot = 0.0;
+                        for (int j = 0; j < D; ++j) dot += load_elem(q_win, qb + j, dtype) * load_elem(k, kb + j, dtype);
+                        s[t] = dot * scale;
+                        if (s[t] > mx) mx = s[t];
+                    }
+                    double den = 0.0;
+                    for (int t = 0; t <= last; ++t) den += exp(s[t] - mx);
+                    for (int t = 0; t < P; ++t) vote[t] += exp(s[t] - mx) / den;
+                }
+            for (int t = 0; t < P; ++t) {
+                double m = vote[t];
+                for (int u = t - half; u <= t + half; ++u)
+                    if (u >= 0 && u < P && vote[u] > m) m = vote[u];
+                cand[t].p = m;
+                cand[t].t = t;
+                if (vote_out) vote_out[((int64_t)b * Hkv + h) * S_max + t] = vote[t];
+                if (pooled_out) pooled_out[((int64_t)b * Hkv + h) * S_max + t] = m;
+            }
+            qsort(cand, (size_t)P, sizeof(tok_t), tok_cmp);
+            for (int r = 0; r < budget - W; ++r) sel[cand[r].t] = 1;
+            for (int t = P; t < S; ++t) sel[t] = 1;
+            int n = 0;
+            for (int t = 0; t < S; ++t) if (sel[t]) kt[n++] = t;
+            free(vote); free(s); free(cand); free(sel);
+        }
+    return err;
+}

@@ -1,0 +1,324 @@
+"""Pins for the CPU oracle: checks against what the paper and the mathematics fix.
+
+Nothing here re-types the oracle's own loops: every expected value is a closed
+form, a brute-force enumeration, a textbook routine written independently in
+NumPy, or the hand-worked fixture under tests/golden/.
+"""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def dense_attention(q, K, V, scale=None):
+    """Textbook softmax(q K^T / sqrt(D)) V for one head, float64 (Sec. Preliminaries)."""
+    q, K, V = np.asarray(q, np.float64), np.asarray(K, np.float64), np.asarray(V, np.float64)
+    s = K @ q * (scale if scale else 1.0 / math.sqrt(K.shape[1]))
+    e = np.exp(s - s.max())
+    return (e / e.sum()) @ V, s.max() + math.log(e.sum())
+
+
+def rand_case(rng, B=1, Hq=1, Hkv=1, W=4, D=8, S=5, scale=1.0):
+    q_win = rng.standard_normal((B, Hq, W, D)).astype(np.float32) * scale
+    k = rng.standard_normal((B, Hkv, S, D)).astype(np.float32) * scale
+    v = rng.standard_normal((B, Hkv, S, D)).astype(np.float32)
+    q = rng.standard_normal((B, Hq, D)).astype(np.float32)
+    return q_win, k, v, q
+
+
+def bits_of(mask_row, D):
+    return [j for j in range(D) if (int(mask_row[j // 32]) >> (j % 32)) & 1]
+
+
+# ---------------------------------------------------------------- hand-worked fixture
+def test_hand_example_whole_chain():
+    g = json.load(open(os.path.join(GOLD, "hand_example.json")))
+    D, T = g["D"], g["T"]
+    q_win = np.array(g["q_win"], np.float32).reshape(1, 1, g["W"], D)
+    k = np.array(g["k"], np.float32).reshape(1, 1, 3, D)
+    v = np.zeros((1, 1, 3, D), np.float32)
+    v[0, 0, :, :2] = np.array(g["v"], np.float32)
+    q = np.array(g["q"], np.float32).reshape(1, 1, D)
+    qbar, a = oracle.window_mean(q_win, 1)
+    assert np.array_equal(qbar[0, 0], np.array(g["qbar"], np.float32))
+    assert np.array_equal(a[0, 0], np.abs(np.array(g["qbar"], np.float32)))
+    c = oracle.compress(k, [3], T, a, want_idx=True, want_saliency=True)
+    assert np.array_equal(c["saliency"][0, 0], np.array(g["saliency"], np.float32))
+    assert [int(x) for x in c["mask"][0, 0, :, 0]] == g["mask"]
+    assert np.array_equal(c["mu"][0, 0], np.array(g["mu"], np.float32))
+    for path in (0, 1):
+        out, lse, sc = oracle.decode_attn(q, k, v, [3], c["mask"], c["mu"], a, path=path, want_scores=True)
+        assert np.allclose(sc[0, 0], g["scores"], rtol=0, atol=5e-8)
+        assert np.allclose(out[0, 0, :2], g["out"], rtol=0, atol=1e-7)   # float32 output
+    # the recovered key rows of the fixture reproduce its scores (checks the fixture itself)
+    kr = np.array(g["k_recovered"])
+    assert np.allclose(kr @ np.array(g["q"]) / math.sqrt(D), g["scores"], atol=5e-8)
+
+
+# ---------------------------------------------------------------- window mean
+def test_window_mean_pools_group_queries_exactly():
+    rng = np.random.default_rng(1)
+    B, Hq, Hkv, W, D = 2, 6, 2, 8, 16
+    # small integers / 8: sums are exact in any order, so the mean has one right answer
+    q_win = (rng.integers(-40, 41, (B, Hq, W, D)) / 8.0).astype(np.float32)
+    qbar, a = oracle.window_mean(q_win, Hkv, eps=0.3)
+    G = Hq // Hkv
+    want = q_win.astype(np.float64).reshape(B, Hkv, G, W, D).sum(axis=(2, 3)) / (G * W)
+    assert np.array_equal(qbar, want.astype(np.float32))
+    assert np.array_equal(a, np.maximum(np.abs(want.astype(np.float32)), np.float32(0.3)))
+    assert (a >= np.float32(0.3)).all() and (np.abs(qbar) < 0.3).any()   # the floor is exercised
+
+
+def test_window_mean_bf16_input_is_widened_exactly():
+    torch = pytest.importorskip("torch")
+    x = torch.tensor([[[[1.0, -2.5, 0.15625, 3.0]] * 2]], dtype=torch.bfloat16)   # [1,1,2,4]
+    qbar, a = oracle.window_mean(x, 1)
+    assert np.array_equal(qbar[0, 0], np.array([1.0, -2.5, 0.15625, 3.0], np.float32))
+
+
+# ---------------------------------------------------------------- selection (Eq. cal)
+@pytest.mark.parametrize("D", [8, 10])
+def test_top_t_equals_brute_force_argmax_of_linear_objective(D):
+    rng = np.random.default_rng(D)
+    q_win, k, v, q = rand_case(rng, D=D, S=6)
+    _, a = oracle.window_mean(q_win, 1)
+    w = (a[0, 0][None, :] * np.abs(k[0, 0])).astype(np.float64)       # saliency, Sec. Problem Formulation
+    for T in range(1, D + 1):
+        c = oracle.compress(k, [6], T, a, want_idx=True)
+        for t in range(6):
+            best = max(itertools.combinations(range(D), T), key=lambda s: sum(w[t, j] for j in s))
+            assert bits_of(c["mask"][0, 0, t], D) == list(best)
+            assert list(c["kept_idx"][0, 0, t]) == list(best)
+
+
+def test_ties_keep_lower_channel():
+    D, T = 8, 3
+    a = np.ones((1, 1, D), np.float32)
+    k = np.array([[[[2, 1, 1, 1, 1, 0.5, 2, 1]]]], np.float32)        # w: two 2s, five 1s
+    c = oracle.compress(k, [1], T, a)
+    assert bits_of(c["mask"][0, 0, 0], D) == [0, 1, 6]                 # 2s, then the FIRST of the 1s
+    k2 = np.ones((1, 1, 1, D), np.float32)
+    c2 = oracle.compress(k2, [1], 5, a)
+    assert bits_of(c2["mask"][0, 0, 0], D) == [0, 1, 2, 3, 4]
+
+
+def test_popcount_separation_and_mu_on_random_heads():
+    rng = np.random.default_rng(3)
+    B, Hq, Hkv, W, D, S = 2, 4, 2, 8, 128, 40
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S, scale=2.0)
+    _, a = oracle.window_mean(q_win, Hkv)
+    for T in (1, 25, 64, 127, 128):
+        c = oracle.compress(k, [S, S - 7], T, a, want_idx=True, want_saliency=True)
+        for b, h, t in itertools.product(range(B), range(Hkv), range(S)):
+            kept = bits_of(c["mask"][b, h, t], D)
+            if t >= [S, S - 7][b]:
+                assert kept == [] and c["mu"][b, h, t] == 0
+                continue
+            assert len(kept) == T                                       # sum_j z_j = T
+            assert kept == sorted(kept) == list(c["kept_idx"][b, h, t])
+            w = a[b, h] * np.abs(k[b, h, t])                            # fp32 product
+            assert np.array_equal(w, c["saliency"][b, h, t])
+            pruned = [j for j in range(D) if j not in kept]
+            if pruned:
+                assert w[kept].min() >= w[pruned].max()
+                assert np.isclose(c["mu"][b, h, t], w[pruned].astype(np.float64).mean(), rtol=1e-6)
+            else:
+                assert c["mu"][b, h, t] == 0
+
+
+def test_all_channel_statistics_are_population_moments():
+    rng = np.random.default_rng(5)
+    q_win, k, v, q = rand_case(rng, D=32, S=9)
+    _, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [9], 16, a, want_saliency=True, want_stats=True)
+    w = c["saliency"][0, 0].astype(np.float64)
+    assert np.allclose(c["mu_all"][0, 0], w.mean(axis=1), rtol=1e-6)
+    assert np.allclose(c["sigma_all"][0, 0], w.std(axis=1), rtol=1e-6)   # 1/|C| normalisation
+
+
+def test_strided_token_major_layout_matches_head_major():
+    rng = np.random.default_rng(6)
+    q_win, k, v, q = rand_case(rng, B=2, Hq=4, Hkv=2, D=16, S=7)
+    _, a = oracle.window_mean(q_win, 2)
+    c1 = oracle.compress(k, [7, 5], 6, a)
+    k_tm = np.ascontiguousarray(k.transpose(0, 2, 1, 3)).transpose(0, 2, 1, 3)   # [B,S,H,D] storage
+    v_tm = np.ascontiguousarray(v.transpose(0, 2, 1, 3)).transpose(0, 2, 1, 3)
+    assert k_tm.strides != k.strides
+    c2 = oracle.compress(k_tm, [7, 5], 6, a)
+    assert np.array_equal(c1["mask"], c2["mask"]) and np.array_equal(c1["mu"], c2["mu"])
+    o1, l1 = oracle.decode_attn(q, k, v, [7, 5], c1["mask"], c1["mu"], a)
+    o2, l2 = oracle.decode_attn(q, k_tm, v_tm, [7, 5], c1["mask"], c1["mu"], a)
+    assert np.array_equal(o1, o2) and np.array_equal(l1, l2)
+
+
+# ---------------------------------------------------------------- recovery + attention
+def test_ratio_zero_is_dense_attention_with_gqa_mapping():
+    rng = np.random.default_rng(7)
+    B, Hq, Hkv, W, D, S = 2, 6, 2, 4, 32, 50
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S)
+    lens = [S, 31]
+    _, a = oracle.window_mean(q_win, Hkv)
+    c = oracle.compress(k, lens, D, a)
+    assert (c["mu"] == 0).all()
+    for b in range(B):
+        assert (c["mask"][b, :, :lens[b]] == 0xFFFFFFFF).all()
+    for path in (0, 1):
+        out, lse = oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, path=path)
+        for b, i in itertools.product(range(B), range(Hq)):
+            h = i // (Hq // Hkv)
+            want, want_lse = dense_attention(q[b, i], k[b, h, :lens[b]], v[b, h, :lens[b]])
+            assert np.allclose(out[b, i], want, rtol=0, atol=1e-6)
+            assert np.isclose(lse[b, i], want_lse, rtol=0, atol=1e-5)
+
+
+def test_zero_fill_mode_equals_dense_attention_on_masked_keys():
+    rng = np.random.default_rng(8)
+    q_win, k, v, q = rand_case(rng, B=1, Hq=2, Hkv=1, W=4, D=64, S=33)
+    _, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [33], 20, a)
+    dense_mask = np.array([[(int(c["mask"][0, 0, t, j // 32]) >> (j % 32)) & 1 for j in range(64)]
+                           for t in range(33)], np.float64)
+    out, lse = oracle.decode_attn(q, k, v, [33], c["mask"], np.zeros_like(c["mu"]), a)
+    for i in range(2):
+        want, _ = dense_attention(q[0, i], k[0, 0] * dense_mask, v[0, 0])
+        assert np.allclose(out[0, i], want, atol=1e-6)
+
+
+def test_mass_preservation_of_recovered_entries():
+    """sum over pruned j of |q-bar_j| * k~_j equals the pruned saliency mass (D-T) mu."""
+    rng = np.random.default_rng(9)
+    D, S, T = 32, 12, 10
+    q_win, k, v, _ = rand_case(rng, W=6, D=D, S=S)
+    qbar, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [S], T, a, want_saliency=True)
+    # probe query = a itself, scale 1: scores are sum_kept a_j k_j + sum_pruned a_j (mu/a_j)
+    _, _, sc = oracle.decode_attn(a.reshape(1, 1, D), k, v, [S], c["mask"], c["mu"], a,
+                                  scale=1.0, want_scores=True)
+    for t in range(S):
+        kept = bits_of(c["mask"][0, 0, t], D)
+        pruned = [j for j in range(D) if j not in kept]
+        kept_part = float((a[0, 0, kept].astype(np.float64) * k[0, 0, t, kept]).sum())
+        pruned_mass = float(c["saliency"][0, 0, t, pruned].astype(np.float64).sum())
+        assert np.isclose(sc[0, 0, t] - kept_part, pruned_mass, rtol=1e-6)
+        assert np.isclose(pruned_mass, (D - T) * float(c["mu"][0, 0, t]), rtol=1e-6)
+
+
+@pytest.mark.parametrize("T", [1, 5, 16, 31])
+def test_positive_case_collapses_to_dense_attention_for_every_ratio(T):
+    """q-bar > 0, K >= 0, one head, decode query = q-bar: q.K~ = sum_j w_j = q-bar.K for every T."""
+    rng = np.random.default_rng(10 + T)
+    D, S, W = 32, 20, 4
+    base = (rng.integers(1, 64, D) / 16.0).astype(np.float32)            # exactly representable
+    q_win = np.broadcast_to(base, (1, 1, W, D)).copy()                    # mean == base exactly
+    k = (rng.integers(0, 256, (1, 1, S, D)) / 32.0).astype(np.float32)
+    v = rng.standard_normal((1, 1, S, D)).astype(np.float32)
+    qbar, a = oracle.window_mean(q_win, 1)
+    assert np.array_equal(qbar[0, 0], base)
+    c = oracle.compress(k, [S], T, a)
+    want, want_lse = dense_attention(base, k[0, 0], v[0, 0])
+    for path in (0, 1):
+        out, lse = oracle.decode_attn(base.reshape(1, 1, D), k, v, [S], c["mask"], c["mu"], a, path=path)
+        assert np.allclose(out[0, 0], want, atol=2e-6)
+        assert np.isclose(lse[0, 0], want_lse, atol=1e-5)
+
+
+def test_two_score_paths_agree_and_splits_merge_by_lse():
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, W, D, S = 1, 4, 2, 8, 128, 200
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S, scale=1.5)
+    _, a = oracle.window_mean(q_win, Hkv)
+    c = oracle.compress(k, [S], 40, a)
+    o0, l0, s0 = oracle.decode_attn(q, k, v, [S], c["mask"], c["mu"], a, path=0, want_scores=True)
+    o1, l1, s1 = oracle.decode_attn(q, k, v, [S], c["mask"], c["mu"], a, path=1, want_scores=True)
+    assert np.allclose(s0, s1, rtol=1e-12, atol=1e-12)
+    assert np.allclose(o0, o1, atol=1e-7)
+    # split the tokens 77 | 123, attend separately, merge with log-sum-exp weights
+    cut = 77
+    parts = []
+    for lo, hi in ((0, cut), (cut, S)):
+        o, l = oracle.decode_attn(q, k[:, :, lo:hi], v[:, :, lo:hi], [hi - lo],
+                                  np.ascontiguousarray(c["mask"][:, :, lo:hi]),
+                                  np.ascontiguousarray(c["mu"][:, :, lo:hi]), a)
+        parts.append((o.astype(np.float64), l.astype(np.float64)))
+    m = np.maximum(parts[0][1], parts[1][1])
+    w0, w1 = np.exp(parts[0][1] - m), np.exp(parts[1][1] - m)
+    merged = (parts[0][0] * w0[..., None] + parts[1][0] * w1[..., None]) / (w0 + w1)[..., None]
+    assert np.allclose(merged, o0, atol=2e-6)
+    assert np.allclose(m + np.log(w0 + w1), l0, atol=1e-5)
+
+
+def test_scale_argument_and_default():
+    rng = np.random.default_rng(12)
+    q_win, k, v, q = rand_case(rng, D=16, S=6)
+    _, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [6], 16, a)
+    o_def, _ = oracle.decode_attn(q, k, v, [6], c["mask"], c["mu"], a)
+    o_exp, _ = oracle.decode_attn(q, k, v, [6], c["mask"], c["mu"], a, scale=0.25)   # 1/sqrt(16)
+    assert np.array_equal(o_def, o_exp)
+    o_one, _ = oracle.decode_attn(q, k, v, [6], c["mask"], c["mu"], a, scale=1.0)
+    want, _ = dense_attention(q[0, 0], k[0, 0], v[0, 0], scale=1.0)
+    assert np.allclose(o_one[0, 0], want, atol=1e-6)
+
+
+def test_empty_sequence_gives_zero_output():
+    rng = np.random.default_rng(13)
+    q_win, k, v, q = rand_case(rng, B=2, D=16, S=4)
+    _, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [0, 4], 8, a)
+    out, lse = oracle.decode_attn(q, k, v, [0, 4], c["mask"], c["mu"], a)
+    assert (out[0] == 0).all() and np.isneginf(lse[0]).all() and np.isfinite(out[1]).all()
+
+
+def test_memory_accounting_of_kept_values():
+    """Kept key values are T/D of the dense keys; at ratio 0.8 K+V values are 60 % (a 40 % cut)."""
+    from paper_2508_15212_b200.inputs import keep_count
+    D = 128
+    assert keep_count(D, 0.5) == 64 and keep_count(D, 0.8) == 25       # floor((1-lambda) D)
+    assert keep_count(D, 0.3) == 89 and keep_count(D, 0.7) == 38 and keep_count(D, 0.0) == 128
+    lam = 0.8
+    assert math.isclose(((1 - lam) * D + D) / (2 * D), 0.6)
+
+
+# ---------------------------------------------------------------- eviction (own invariants only)
+def test_eviction_identity_budget_and_window_always_kept():
+    rng = np.random.default_rng(14)
+    B, Hq, Hkv, W, D, S = 1, 4, 2, 4, 16, 40
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S)
+    kept, n = oracle.evict(q_win, k, [S], budget=64, pool=7)
+    assert n[0] == S and (kept[0, :, :S] == np.arange(S)).all() and (kept[0, :, S:] == -1).all()
+    kept, n = oracle.evict(q_win, k, [S], budget=12, pool=7)
+    assert n[0] == 12
+    for h in range(Hkv):
+        row = list(kept[0, h])
+        assert row == sorted(row) and len(set(row)) == 12
+        assert row[-W:] == list(range(S - W, S))
+
+
+def test_eviction_pool_one_is_plain_top_k_of_causal_window_votes():
+    rng = np.random.default_rng(15)
+    B, Hq, Hkv, W, D, S, budget = 1, 2, 1, 3, 8, 17, 9
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S)
+    kept, n, vote, pooled = oracle.evict(q_win, k, [S], budget=budget, pool=1, want_votes=True)
+    P = S - W
+    want_vote = np.zeros(P)
+    for g in range(Hq):
+        for w in range(W):
+            last = P + w
+            s = k[0, 0, :last + 1].astype(np.float64) @ q_win[0, g, w].astype(np.float64) / math.sqrt(D)
+            e = np.exp(s - s.max())
+            want_vote += (e / e.sum())[:P]
+    assert np.allclose(vote[0, 0, :P], want_vote, rtol=1e-12)
+    assert np.array_equal(pooled[0, 0, :P], vote[0, 0, :P])
+    top = sorted(sorted(range(P), key=lambda t: (-want_vote[t], t))[:budget - W])
+    assert list(kept[0, 0]) == top + list(range(P, S))
+    # pooling: each pooled value is the max of its clamped 5-neighbourhood
+    _, _, vote5, pooled5 = oracle.evict(q_win, k, [S], budget=budget, pool=5, want_votes=True)
+    for t in range(P):
+        assert pooled5[0, 0, t] == vote5[0, 0, max(0, t - 2):min(P, t + 3)].max()
