@@ -1,0 +1,187 @@
+/*
+ * spark.h -- C ABI of the SparK hot path on one NVIDIA B200 (sm_100a).
+ *
+ * SparK prunes the key cache per token along the channel axis and restores the
+ * pruned entries while the decode query is scored.  Two calls carry the method:
+ *
+ *   spark_compress      observation-window queries + full K/V  ->  packed cache
+ *   spark_decode_attn   decode query + packed cache            ->  attention output
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless marked
+ *     "host".  The library allocates nothing and keeps no state between calls.
+ *   - Work is enqueued on the caller's stream (`spark_stream_t` is a
+ *     `cudaStream_t`); nothing synchronises except spark_read_status.
+ *   - Errors the host can see (null pointers, shapes, sizes) are returned as a
+ *     spark_status BEFORE any launch.  Errors only the device can see (a page
+ *     id outside the pool, a bounded wait that ran out) are recorded in the
+ *     status word at the start of the workspace and the kernel returns without
+ *     touching the bad address; read them with spark_read_status.
+ *   - head_dim must be 128, page_tokens 16, 1 <= n_q_heads / n_kv_heads <= 8.
+ *
+ * Packed cache.  The cache is a pool of fixed-size pages.  One page holds
+ * `page_tokens` consecutive tokens of ONE KV head of one sequence:
+ *     kept key values (ascending channel order) | 128-bit channel mask per token
+ *     | mu_pruned per token (fp32) | dense value rows
+ * `block_table[b][h][i]` is the pool index of the page with tokens
+ * [16 i, 16 i + 16) of sequence b, KV head h.  The byte layout inside a page is
+ * private to the library (spark_page_bytes gives its size; spark_unpack_pages
+ * turns pages back into logical arrays).  Slots of a page past the end of the
+ * sequence are zero.
+ */
+#ifndef SPARK_H_
+#define SPARK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *spark_stream_t;            /* a cudaStream_t; NULL is the legacy default stream */
+
+typedef enum {
+    SPARK_OK = 0,
+    SPARK_ERR_NULL = 1,                  /* a required pointer is NULL                        */
+    SPARK_ERR_BAD_SHAPE = 2,             /* inconsistent or out-of-range sizes                */
+    SPARK_ERR_UNSUPPORTED = 3,           /* head_dim != 128, page_tokens != 16, dtype, G > 8  */
+    SPARK_ERR_WORKSPACE = 4,             /* workspace missing, misaligned or too small        */
+    SPARK_ERR_CUDA = 5,                  /* a CUDA runtime call failed (launch, attribute)    */
+    SPARK_ERR_DEVICE_BOUNDS = 6,         /* device saw a page id / length out of range        */
+    SPARK_ERR_DEVICE_TIMEOUT = 7         /* a bounded device-side wait ran out                */
+} spark_status;
+
+typedef enum { SPARK_F32 = 0, SPARK_BF16 = 1 } spark_dtype;
+
+typedef struct {
+    int32_t batch;          /* B, sequences                                                   */
+    int32_t n_q_heads;      /* Hq                                                             */
+    int32_t n_kv_heads;     /* Hkv; query head i reads KV head i / (Hq / Hkv)                 */
+    int32_t head_dim;       /* D = 128                                                        */
+    int32_t window;         /* W, observation-window queries per query head                   */
+    int32_t keep;           /* T, kept key channels per token, 1..D                           */
+    int32_t page_tokens;    /* 16                                                             */
+    int32_t dtype;          /* spark_dtype of q, k, v and of the packed values                */
+    int32_t token_budget;   /* 0: no eviction; else tokens kept per KV head, window included  */
+    int32_t pool_kernel;    /* odd max-pool width of the eviction votes (7); budget > 0 only  */
+    float   qnorm_eps;      /* floor of |mean window query|; 0 selects 1e-12                  */
+    float   softmax_scale;  /* 0 selects 1/sqrt(head_dim)                                     */
+    int64_t n_pool_pages;   /* pages in the pool; every block-table entry must be below it    */
+} spark_params;
+
+/* T = floor((1 - ratio) * head_dim): the paper's kept-channel count (Sec. "Problem
+ * Formulation", below Eq. (cal)).  Host only.  Returns -1 for ratio outside [0, 1). */
+int32_t spark_keep_count(int32_t head_dim, double ratio);
+
+/* Bytes of one page for these parameters (uses head_dim, keep, page_tokens, dtype).
+ * Host only.  0 on unsupported parameters. */
+size_t spark_page_bytes(const spark_params *p);
+
+/* Bytes the method itself has to read per token and KV head in one decode step:
+ * kept values + mask + mu_pruned + dense value row (the roofline numerator).  Host only. */
+size_t spark_algorithmic_bytes_per_token(const spark_params *p);
+
+/* Workspace sizes.  `max_seq_tokens` bounds seq_lens (before eviction).  Either
+ * output pointer may be NULL.  Host only. */
+spark_status spark_workspace_bytes(const spark_params *p, int64_t max_seq_tokens,
+                                   size_t *compress_bytes, size_t *decode_bytes);
+
+/* Zero a workspace.  Must be enqueued once before the first call that uses the
+ * workspace; the calls leave it ready for the next one. */
+spark_status spark_workspace_init(void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
+ * spark_compress -- prefill-side pruning (Sec. "SparK": "Saliency Measurement and
+ * Unstructured Pruning"; statistics of App. "Caching Pruned Channel Statistics").
+ *
+ * For every sequence b and KV head h:
+ *   q-bar[j] = mean of the G*W window queries of the G query heads that share h
+ *   a[j]     = max(|q-bar[j]|, qnorm_eps)                       -> qnorm[b][h][j]
+ *   w[t][j]  = a[j] * |K[t][j]|      one round-to-nearest fp32 multiply
+ *   kept_t   = the `keep` channels of largest w[t][.], lower channel first on ties
+ *   mu[t]    = mean of w[t][j] over the pruned channels (0 when keep == head_dim)
+ * and the page of token t receives K[t][kept_t] (bit-identical, ascending channel
+ * order), the mask, mu[t] and V[t][:].
+ *
+ * With token_budget > 0 the tokens are first reduced per KV head to
+ * min(S_b, token_budget) by observation-window attention votes (softmax of the
+ * window queries against all earlier keys, causal inside the window, summed over
+ * the group and the window, max-pooled with pool_kernel, top-(budget - W) of the
+ * prefix plus the W window tokens, original order); the paper cites this step
+ * from its base eviction method (App. "Implementation") and does not define it.
+ *
+ *   q_win        [B][Hq][W][D] contiguous; the window is the LAST W tokens of each sequence
+ *   k, v         element (b,h,t,j) at b*stride_b + h*stride_h + t*stride_t + j (in elements)
+ *   seq_lens     [B] int32, tokens per sequence (<= max_seq_tokens)
+ *   pages        OUT page pool, n_pool_pages * spark_page_bytes(p) bytes, 16-byte aligned
+ *   block_table  [B][Hkv][max_blocks] int32 pool indices; entries are read for
+ *                i < ceil(packed_len_b / 16)
+ *   qnorm        OUT [B][Hkv][D] fp32
+ *   packed_lens  OUT [B] int32, tokens per KV head after eviction (= seq_lens when budget == 0)
+ *   kept_tokens  OUT optional [B][Hkv][token_budget] int32 original positions (budget > 0), else NULL
+ *   workspace    scratch of at least compress_bytes (spark_workspace_bytes), 256-byte aligned
+ */
+spark_status spark_compress(const spark_params *p,
+                            const void *q_win, const void *k, const void *v,
+                            int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                            const int32_t *seq_lens, int32_t max_seq_tokens,
+                            void *pages, const int32_t *block_table, int32_t max_blocks,
+                            float *qnorm, int32_t *packed_lens, int32_t *kept_tokens,
+                            void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
+ * spark_decode_attn -- one decode step over the packed cache (Sec. "Channel Recovery"
+ * with the degenerate distribution, then the attention of Sec. "Preliminaries").
+ *
+ * For every sequence b and query head i (KV head h = i / G):
+ *   K~[t][j] = K[t][j] if channel j of token t was kept, else mu[t] / a[j]
+ *   s[t]     = softmax_scale * sum_j q[i][j] * K~[t][j]
+ *   out[i]   = sum_t softmax_t(s)[t] * V[t][:]          over t < packed_lens[b]
+ * Accumulation is fp32; the softmax is computed online over token splits that are
+ * merged by their log-sum-exp.  A sequence of length 0 yields out = 0, lse = -inf.
+ *
+ *   q            [B][Hq][D] contiguous, dtype as the cache
+ *   pages, block_table, max_blocks, packed_lens, qnorm   as written by spark_compress
+ *   out          OUT [B][Hq][D] fp32
+ *   lse          OUT optional [B][Hq] fp32, natural-log sum-exp of the scaled scores
+ *   workspace    at least decode_bytes, 256-byte aligned, initialised once by spark_workspace_init
+ */
+spark_status spark_decode_attn(const spark_params *p, const void *q,
+                               const void *pages, const int32_t *block_table, int32_t max_blocks,
+                               const int32_t *packed_lens, const float *qnorm,
+                               float *out, float *lse,
+                               void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
+ * spark_unpack_pages -- pages back to logical arrays (what the paper calls the pruned
+ * key matrix K^, the mask S and mu_pruned; Sec. "Saliency Measurement and Unstructured
+ * Pruning").  For inspection and tests; any output may be NULL.
+ *
+ *   mask   OUT [B][Hkv][max_tokens][4] uint32, bit (j % 32) of word (j / 32) <=> channel j kept
+ *   mu     OUT [B][Hkv][max_tokens] fp32
+ *   vals   OUT [B][Hkv][max_tokens][keep] in the cache dtype, ascending channel order
+ *   v      OUT [B][Hkv][max_tokens][D] in the cache dtype
+ * Rows t >= packed_lens[b] are written as zeros.
+ */
+spark_status spark_unpack_pages(const spark_params *p, const void *pages,
+                                const int32_t *block_table, int32_t max_blocks,
+                                const int32_t *packed_lens, int32_t max_tokens,
+                                uint32_t *mask, float *mu, void *vals, void *v,
+                                spark_stream_t stream);
+
+/* Synchronise `stream` and return the status word of a workspace (SPARK_OK when no
+ * kernel recorded an error).  Debug and tests only. */
+spark_status spark_read_status(const void *workspace, spark_stream_t stream);
+
+/* Number of kernels the last successful spark_decode_attn / spark_compress call of this
+ * thread enqueued (host only; for launch accounting in benchmarks). */
+int32_t spark_last_launch_count(void);
+
+/* Library version: major * 10000 + minor * 100 + patch.  Host only. */
+int32_t spark_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARK_H_ */

@@ -1,0 +1,157 @@
+// C ABI of the SparK library: argument checks, sizes, and dispatch to the kernel launchers.
+#include <math.h>
+
+#include "spark_common.cuh"
+
+using namespace spark;
+
+static thread_local int g_last_launches = 0;
+
+static spark_status check_params(const spark_params* p)
+{
+    if (!p) return SPARK_ERR_NULL;
+    if (p->head_dim != kHeadDim || p->page_tokens != kPageTokens) return SPARK_ERR_UNSUPPORTED;
+    if (p->dtype != SPARK_F32 && p->dtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
+    if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1) return SPARK_ERR_BAD_SHAPE;
+    if (p->n_q_heads % p->n_kv_heads) return SPARK_ERR_BAD_SHAPE;
+    if (p->n_q_heads / p->n_kv_heads > kMaxGroup) return SPARK_ERR_UNSUPPORTED;
+    if (p->batch > kMaxBatch) return SPARK_ERR_UNSUPPORTED;
+    if (p->keep < 1 || p->keep > p->head_dim) return SPARK_ERR_BAD_SHAPE;
+    if (p->n_pool_pages < 1) return SPARK_ERR_BAD_SHAPE;
+    if (p->token_budget < 0) return SPARK_ERR_BAD_SHAPE;
+    if (!(p->qnorm_eps >= 0.f) || !(p->softmax_scale >= 0.f)) return SPARK_ERR_BAD_SHAPE;
+    return SPARK_OK;
+}
+
+extern "C" {
+
+int32_t spark_version(void) { return 100; }
+
+int32_t spark_last_launch_count(void) { return g_last_launches; }
+
+int32_t spark_keep_count(int32_t head_dim, double ratio)
+{
+    if (!(ratio >= 0.0) || !(ratio < 1.0) || head_dim < 1) return -1;
+    // the small offset absorbs binary representation error of ratios whose product is an integer
+    return static_cast<int32_t>(floor((1.0 - ratio) * head_dim + 1e-9));
+}
+
+size_t spark_page_bytes(const spark_params* p)
+{
+    if (!p || p->head_dim != kHeadDim || p->page_tokens != kPageTokens) return 0;
+    if (p->dtype != SPARK_F32 && p->dtype != SPARK_BF16) return 0;
+    if (p->keep < 1 || p->keep > kHeadDim) return 0;
+    return static_cast<size_t>(make_layout(p->dtype, p->keep).page_bytes);
+}
+
+size_t spark_algorithmic_bytes_per_token(const spark_params* p)
+{
+    if (!p || p->keep < 1 || p->keep > p->head_dim) return 0;
+    const size_t e = (p->dtype == SPARK_BF16) ? 2 : 4;
+    return e * p->keep + 16 + 4 + e * p->head_dim;
+}
+
+spark_status spark_workspace_bytes(const spark_params* p, int64_t max_seq_tokens,
+                                   size_t* compress_bytes, size_t* decode_bytes)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (max_seq_tokens < 0) return SPARK_ERR_BAD_SHAPE;
+    if (compress_bytes) *compress_bytes = compress_workspace_bytes(*p, max_seq_tokens);
+    if (decode_bytes) *decode_bytes = decode_workspace_bytes(*p);
+    return SPARK_OK;
+}
+
+spark_status spark_workspace_init(void* workspace, size_t workspace_bytes, spark_stream_t stream)
+{
+    if (!workspace) return SPARK_ERR_NULL;
+    if (workspace_bytes < kWorkspaceHeader || (reinterpret_cast<uintptr_t>(workspace) & 255))
+        return SPARK_ERR_WORKSPACE;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    return SPARK_OK;
+}
+
+spark_status spark_compress(const spark_params* p, const void* q_win, const void* k, const void* v,
+                            int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                            const int32_t* seq_lens, int32_t max_seq_tokens, void* pages,
+                            const int32_t* block_table, int32_t max_blocks, float* qnorm,
+                            int32_t* packed_lens, int32_t* kept_tokens, void* workspace,
+                            size_t workspace_bytes, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!q_win || !k || !v || !seq_lens || !pages || !block_table || !qnorm || !packed_lens || !workspace)
+        return SPARK_ERR_NULL;
+    if (p->window < 1 || max_seq_tokens < 0 || max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
+    if (stride_t < p->head_dim || stride_b < 0 || stride_h < 0) return SPARK_ERR_BAD_SHAPE;
+    if (reinterpret_cast<uintptr_t>(pages) & 15) return SPARK_ERR_BAD_SHAPE;
+    // vector loads of K/V rows need 16-byte aligned rows
+    const int e = (p->dtype == SPARK_BF16) ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(k) & 15) || (reinterpret_cast<uintptr_t>(v) & 15) ||
+        ((stride_b * e) & 15) || ((stride_h * e) & 15) || ((stride_t * e) & 15))
+        return SPARK_ERR_BAD_SHAPE;
+    if (p->token_budget > 0) {
+        if (p->token_budget < p->window || p->pool_kernel < 1 || !(p->pool_kernel & 1))
+            return SPARK_ERR_BAD_SHAPE;
+        if (!kept_tokens) return SPARK_ERR_NULL;
+    }
+    const int64_t max_packed = (p->token_budget > 0 && p->token_budget < max_seq_tokens)
+                                   ? p->token_budget : max_seq_tokens;
+    if ((max_packed + kPageTokens - 1) / kPageTokens > max_blocks) return SPARK_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) ||
+        workspace_bytes < compress_workspace_bytes(*p, max_seq_tokens))
+        return SPARK_ERR_WORKSPACE;
+    int launches = 0;
+    st = launch_compress(*p, q_win, k, v, stride_b, stride_h, stride_t, seq_lens, max_seq_tokens, pages,
+                         block_table, max_blocks, qnorm, packed_lens, kept_tokens, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(stream), &launches);
+    if (st == SPARK_OK) g_last_launches = launches;
+    return st;
+}
+
+spark_status spark_decode_attn(const spark_params* p, const void* q, const void* pages,
+                               const int32_t* block_table, int32_t max_blocks,
+                               const int32_t* packed_lens, const float* qnorm, float* out, float* lse,
+                               void* workspace, size_t workspace_bytes, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!q || !pages || !block_table || !packed_lens || !qnorm || !out || !workspace) return SPARK_ERR_NULL;
+    if (max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
+    if (reinterpret_cast<uintptr_t>(pages) & 15) return SPARK_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < decode_workspace_bytes(*p))
+        return SPARK_ERR_WORKSPACE;
+    int launches = 0;
+    st = launch_decode(*p, q, pages, block_table, max_blocks, packed_lens, qnorm, out, lse, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(stream), &launches);
+    if (st == SPARK_OK) g_last_launches = launches;
+    return st;
+}
+
+spark_status spark_unpack_pages(const spark_params* p, const void* pages, const int32_t* block_table,
+                                int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
+                                uint32_t* mask, float* mu, void* vals, void* v, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!pages || !block_table || !packed_lens) return SPARK_ERR_NULL;
+    if (max_tokens < 0 || max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
+    if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
+        return SPARK_ERR_BAD_SHAPE;
+    return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, mask, mu, vals, v,
+                         static_cast<cudaStream_t>(stream));
+}
+
+spark_status spark_read_status(const void* workspace, spark_stream_t stream)
+{
+    if (!workspace) return SPARK_ERR_NULL;
+    int code = 0;
+    if (cudaMemcpyAsync(&code, workspace, sizeof(int), cudaMemcpyDeviceToHost,
+                        static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARK_ERR_CUDA;
+    return static_cast<spark_status>(code);
+}
+
+}  // extern "C"

@@ -1,0 +1,101 @@
+// Shared declarations of the SparK CUDA library: page layout, status word, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/spark.h"
+
+namespace spark {
+
+constexpr int kHeadDim = 128;        // D
+constexpr int kPageTokens = 16;      // P
+constexpr int kMaskWords = 4;        // 128-bit channel mask per token
+constexpr int kMaxGroup = 8;         // G = Hq / Hkv
+constexpr int kMaxBatch = 1024;      // sequences per call (decode keeps a per-sequence prefix in shared memory)
+constexpr int kMaxCtas = 1024;       // upper bound of the persistent decode grid (sizes the partial-result slots)
+constexpr int kWorkspaceHeader = 256;
+
+// Byte layout of one page (16 tokens of one KV head).  Private to the library.
+//
+//   vals : `rows` rows of 64 bytes.  bf16: row r holds slots 2r and 2r+1 of every token, token p at
+//          byte p*4 (+2 for the odd slot); fp32: row r holds slot r, token p at byte p*4.  Slot s of a
+//          token is its s-th kept channel in ascending channel order.  A row is one 64-byte line for the
+//          16 tokens, so a lane-per-token reader hits 16 distinct banks whatever slot each lane is at.
+//   mask : [16][4] uint32, bit (j % 32) of word (j / 32) set <=> channel j kept
+//   mu   : [16] float, mean saliency of the pruned channels
+//   v    : [16][128] elements, dense value rows
+struct PageLayout {
+    int esize;       // bytes per element (2 bf16, 4 fp32)
+    int keep;        // T
+    int rows;        // ceil(T/2) for bf16, T for fp32
+    int mask_off;
+    int mu_off;
+    int v_off;
+    int page_bytes;
+};
+
+__host__ __device__ inline PageLayout make_layout(int dtype, int keep)
+{
+    PageLayout L;
+    L.esize = (dtype == SPARK_BF16) ? 2 : 4;
+    L.keep = keep;
+    L.rows = (dtype == SPARK_BF16) ? (keep + 1) / 2 : keep;
+    L.mask_off = L.rows * 64;
+    L.mu_off = L.mask_off + kPageTokens * 16;
+    L.v_off = L.mu_off + kPageTokens * 4;
+    L.page_bytes = L.v_off + kPageTokens * kHeadDim * L.esize;
+    return L;
+}
+
+// byte offset of kept slot s of token p inside the vals section
+__host__ __device__ inline int val_offset(int esize, int p, int s)
+{
+    return esize == 2 ? ((s >> 1) * 64 + p * 4 + (s & 1) * 2) : (s * 64 + p * 4);
+}
+
+// Workspace header: word 0 is the status word (first error wins).
+__device__ inline void record_error(int* status, int code)
+{
+    atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(unsigned short h)
+{
+    return __uint_as_float(static_cast<unsigned>(h) << 16);
+}
+
+template <typename E> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int dtype = SPARK_F32;
+    __device__ static float load(const void* p, int64_t i) { return static_cast<const float*>(p)[i]; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int dtype = SPARK_BF16;
+    __device__ static float load(const void* p, int64_t i)
+    {
+        return bf16_bits_to_float(static_cast<const unsigned short*>(p)[i]);
+    }
+};
+
+// ---- host-side launchers implemented in the .cu files -------------------------------------------
+spark_status launch_compress(const spark_params& p, const void* q_win, const void* k, const void* v,
+                             int64_t sb, int64_t sh, int64_t st, const int32_t* seq_lens,
+                             int32_t max_seq_tokens, void* pages, const int32_t* block_table,
+                             int32_t max_blocks, float* qnorm, int32_t* packed_lens, int32_t* kept_tokens,
+                             void* workspace, size_t workspace_bytes, cudaStream_t stream, int* launches);
+
+spark_status launch_unpack(const spark_params& p, const void* pages, const int32_t* block_table,
+                           int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
+                           uint32_t* mask, float* mu, void* vals, void* v, cudaStream_t stream);
+
+spark_status launch_decode(const spark_params& p, const void* q, const void* pages,
+                           const int32_t* block_table, int32_t max_blocks, const int32_t* packed_lens,
+                           const float* qnorm, float* out, float* lse, void* workspace,
+                           size_t workspace_bytes, cudaStream_t stream, int* launches);
+
+size_t decode_workspace_bytes(const spark_params& p);
+size_t compress_workspace_bytes(const spark_params& p, int64_t max_seq_tokens);
+
+}  // namespace spark

@@ -1,0 +1,333 @@
+// Prefill-side kernels: window-mean query norm, per-token top-T channel selection + page packing,
+// and the inverse (pages -> logical arrays).
+//
+// Method (paper sections): the mean window query replaces per-token queries (Sec. "SparK"); the
+// saliency of channel j of token t is w = |q-bar_j| * |K[t][j]| (Sec. "Problem Formulation"); the T
+// channels of largest w are kept (Eq. (cal)); the mean saliency of the pruned channels is cached per
+// token (App. "Caching Pruned Channel Statistics").
+#include "spark_common.cuh"
+
+namespace spark {
+
+constexpr unsigned kFullMask = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------------
+// a[b][h][j] = max(|mean over the G*W window queries of the group|, eps).
+// One thread per channel; the sum runs in double over (g outer, w inner), so the rounded mean does
+// not depend on launch shape.  Thread 0 of the first head also publishes packed_lens when there is
+// no eviction step.
+// ------------------------------------------------------------------------------------------------
+template <typename E>
+__global__ void __launch_bounds__(kHeadDim)
+window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, float eps,
+                    float* __restrict__ qnorm, const int32_t* __restrict__ seq_lens,
+                    int32_t* __restrict__ packed_lens, int max_seq_tokens, int* status)
+{
+    const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
+    const int G = Hq / Hkv;
+    double acc = 0.0;
+    for (int g = 0; g < G; ++g) {
+        const int64_t base = ((static_cast<int64_t>(b) * Hq + (h * G + g)) * W) * kHeadDim + j;
+        for (int w = 0; w < W; ++w)
+            acc += static_cast<double>(Elem<E>::load(q_win, base + static_cast<int64_t>(w) * kHeadDim));
+    }
+    const float m = static_cast<float>(acc / static_cast<double>(G * W));
+    qnorm[(static_cast<int64_t>(b) * Hkv + h) * kHeadDim + j] = fmaxf(fabsf(m), eps);
+    if (packed_lens && h == 0 && j == 0) {
+        int len = seq_lens[b];
+        if (len < 0 || len > max_seq_tokens) {
+            record_error(status, SPARK_ERR_DEVICE_BOUNDS);
+            len = len < 0 ? 0 : max_seq_tokens;
+        }
+        packed_lens[b] = len;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// One CTA builds one page (16 tokens of one KV head) in shared memory and writes it out with
+// coalesced 16-byte stores.  One warp per token, two rounds; a lane owns channels 4*lane .. 4*lane+3.
+//
+// Selection is exact: the saliency is one __fmul_rn, its bit pattern (non-negative float) is an
+// order-preserving 31-bit key, the T-th largest key is found by a bitwise radix descent with warp
+// ballots, and keys equal to it are admitted in ascending channel order until T channels are kept.
+// ------------------------------------------------------------------------------------------------
+struct CompressArgs {
+    const void* k;
+    const void* v;
+    int64_t sb, sh, st;
+    const int32_t* lens;          // tokens per sequence AFTER eviction (packed lens)
+    const int32_t* gather;        // optional [B][Hkv][gather_stride] source token positions
+    int gather_stride;
+    const float* qnorm;
+    unsigned char* pages;
+    const int32_t* block_table;
+    int max_blocks;
+    int Hkv;
+    int keep;
+    int64_t n_pool_pages;
+    PageLayout L;
+    int* status;
+};
+
+template <typename E>
+__global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
+{
+    extern __shared__ __align__(16) unsigned char image[];
+    const int blk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int len = A.lens[b];
+    if (blk * kPageTokens >= len) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const PageLayout L = A.L;
+    const int T = A.keep;
+    constexpr bool kBf16 = (sizeof(E) == 2);
+
+    for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(image)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    const float4 a4 = reinterpret_cast<const float4*>(
+        A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
+    const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+    const unsigned lt = (1u << lane) - 1u;
+
+    for (int p = warp; p < kPageTokens; p += 8) {
+        const int t = blk * kPageTokens + p;
+        if (t >= len) continue;                                   // warp-uniform
+        const int src_t = A.gather
+            ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
+        const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
+                            static_cast<int64_t>(src_t) * A.st + lane * 4;
+        unsigned raw[4];
+        float kf[4];
+        if (kBf16) {
+            const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.k) + row);
+            const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.v) + row);
+            raw[0] = kk.x & 0xffffu; raw[1] = kk.x >> 16; raw[2] = kk.y & 0xffffu; raw[3] = kk.y >> 16;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i] << 16);
+            *reinterpret_cast<uint2*>(image + L.v_off + p * (kHeadDim * 2) + lane * 8) = vv;
+        } else {
+            const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.k) + row);
+            const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.v) + row);
+            raw[0] = kk.x; raw[1] = kk.y; raw[2] = kk.z; raw[3] = kk.w;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
+            *reinterpret_cast<uint4*>(image + L.v_off + p * (kHeadDim * 4) + lane * 16) = vv;
+        }
+        float w[4];
+        unsigned key[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
+            key[i] = __float_as_uint(w[i]);
+        }
+        // T-th largest key by radix descent
+        unsigned thr = 0;
+        for (int bit = 30; bit >= 0; --bit) {
+            const unsigned cand = thr | (1u << bit);
+            int cnt = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cnt += __popc(__ballot_sync(kFullMask, key[i] >= cand));
+            if (cnt >= T) thr = cand;
+        }
+        unsigned eqb[4];
+        int c_gt = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            c_gt += __popc(__ballot_sync(kFullMask, key[i] > thr));
+            eqb[i] = __ballot_sync(kFullMask, key[i] == thr);
+        }
+        const int need_eq = T - c_gt;
+        int rank = 0;                                            // equal keys on lower channels
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rank += __popc(eqb[i] & lt);
+        bool kept[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const bool eq = key[i] == thr;
+            kept[i] = key[i] > thr || (eq && rank < need_eq);
+            rank += eq ? 1 : 0;
+        }
+        // slot of each kept channel = kept channels below it
+        int slot = 0;
+        unsigned nib = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            slot += __popc(__ballot_sync(kFullMask, kept[i]) & lt);
+            nib |= kept[i] ? (1u << i) : 0u;
+        }
+        double pruned = 0.0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (kept[i]) {
+                unsigned char* dst = image + val_offset(L.esize, p, slot);
+                if (kBf16) *reinterpret_cast<unsigned short*>(dst) = static_cast<unsigned short>(raw[i]);
+                else *reinterpret_cast<unsigned*>(dst) = raw[i];
+                ++slot;
+            } else {
+                pruned += static_cast<double>(w[i]);
+            }
+        }
+        unsigned word = nib << (4 * (lane & 7));
+        word |= __shfl_xor_sync(kFullMask, word, 1);
+        word |= __shfl_xor_sync(kFullMask, word, 2);
+        word |= __shfl_xor_sync(kFullMask, word, 4);
+        if ((lane & 7) == 0)
+            reinterpret_cast<unsigned*>(image + L.mask_off)[p * kMaskWords + (lane >> 3)] = word;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
+        if (lane == 0)
+            reinterpret_cast<float*>(image + L.mu_off)[p] =
+                (T < kHeadDim) ? static_cast<float>(pruned / static_cast<double>(kHeadDim - T)) : 0.f;
+    }
+    __syncthreads();
+
+    const int page_id = A.block_table[(static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk];
+    if (page_id < 0 || page_id >= A.n_pool_pages) {
+        if (threadIdx.x == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(A.pages + static_cast<int64_t>(page_id) * L.page_bytes);
+    for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
+        dst[i] = reinterpret_cast<const uint4*>(image)[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// pages -> logical arrays
+// ------------------------------------------------------------------------------------------------
+struct UnpackArgs {
+    const unsigned char* pages;
+    const int32_t* block_table;
+    int max_blocks;
+    const int32_t* lens;
+    int max_tokens;
+    int Hkv;
+    int64_t n_pool_pages;
+    PageLayout L;
+    uint32_t* mask;
+    float* mu;
+    void* vals;
+    void* v;
+};
+
+__global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
+{
+    const int blk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const PageLayout L = A.L;
+    const int T = L.keep;
+    int len = A.lens[b];
+    len = len < 0 ? 0 : (len > A.max_tokens ? A.max_tokens : len);
+    const int64_t unit = static_cast<int64_t>(b) * A.Hkv + h;
+    const unsigned char* page = nullptr;
+    if (blk * kPageTokens < len) {
+        const int id = A.block_table[unit * A.max_blocks + blk];
+        if (id >= 0 && id < A.n_pool_pages) page = A.pages + static_cast<int64_t>(id) * L.page_bytes;
+    }
+    const int t0 = blk * kPageTokens;
+    const int64_t row0 = unit * A.max_tokens + t0;
+    if (A.mask)
+        for (int i = threadIdx.x; i < kPageTokens * kMaskWords; i += blockDim.x) {
+            const int p = i / kMaskWords;
+            if (t0 + p >= A.max_tokens) continue;
+            A.mask[(row0 + p) * kMaskWords + (i % kMaskWords)] =
+                (page && t0 + p < len) ? reinterpret_cast<const unsigned*>(page + L.mask_off)[i] : 0u;
+        }
+    if (A.mu)
+        for (int p = threadIdx.x; p < kPageTokens; p += blockDim.x) {
+            if (t0 + p >= A.max_tokens) continue;
+            A.mu[row0 + p] = (page && t0 + p < len) ? reinterpret_cast<const float*>(page + L.mu_off)[p] : 0.f;
+        }
+    if (A.vals)
+        for (int i = threadIdx.x; i < kPageTokens * T; i += blockDim.x) {
+            const int p = i / T, s = i % T;
+            if (t0 + p >= A.max_tokens) continue;
+            const bool live = page && t0 + p < len;
+            const int64_t o = (row0 + p) * T + s;
+            if (L.esize == 2)
+                static_cast<unsigned short*>(A.vals)[o] =
+                    live ? *reinterpret_cast<const unsigned short*>(page + val_offset(2, p, s)) : 0;
+            else
+                static_cast<unsigned*>(A.vals)[o] =
+                    live ? *reinterpret_cast<const unsigned*>(page + val_offset(4, p, s)) : 0u;
+        }
+    if (A.v)
+        for (int i = threadIdx.x; i < kPageTokens * kHeadDim; i += blockDim.x) {
+            const int p = i / kHeadDim;
+            if (t0 + p >= A.max_tokens) continue;
+            const bool live = page && t0 + p < len;
+            const int64_t o = (row0 + p) * kHeadDim + (i % kHeadDim);
+            if (L.esize == 2)
+                static_cast<unsigned short*>(A.v)[o] =
+                    live ? reinterpret_cast<const unsigned short*>(page + L.v_off)[i] : 0;
+            else
+                static_cast<unsigned*>(A.v)[o] = live ? reinterpret_cast<const unsigned*>(page + L.v_off)[i] : 0u;
+        }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+size_t compress_workspace_bytes(const spark_params& p, int64_t max_seq_tokens)
+{
+    size_t bytes = kWorkspaceHeader;
+    (void)max_seq_tokens;
+    (void)p;
+    return bytes;
+}
+
+spark_status launch_compress(const spark_params& p, const void* q_win, const void* k, const void* v,
+                             int64_t sb, int64_t sh, int64_t st, const int32_t* seq_lens,
+                             int32_t max_seq_tokens, void* pages, const int32_t* block_table,
+                             int32_t max_blocks, float* qnorm, int32_t* packed_lens, int32_t* kept_tokens,
+                             void* workspace, size_t workspace_bytes, cudaStream_t stream, int* launches)
+{
+    (void)workspace_bytes;
+    (void)kept_tokens;
+    if (p.token_budget > 0) return SPARK_ERR_UNSUPPORTED;
+    int* status = static_cast<int*>(workspace);
+    const float eps = p.qnorm_eps > 0.f ? p.qnorm_eps : 1e-12f;
+    const dim3 qgrid(p.n_kv_heads, p.batch);
+    if (p.dtype == SPARK_BF16)
+        window_qnorm_kernel<__nv_bfloat16><<<qgrid, kHeadDim, 0, stream>>>(
+            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, packed_lens, max_seq_tokens, status);
+    else
+        window_qnorm_kernel<float><<<qgrid, kHeadDim, 0, stream>>>(
+            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, packed_lens, max_seq_tokens, status);
+    ++*launches;
+    if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
+
+    const int n_blocks = (max_seq_tokens + kPageTokens - 1) / kPageTokens;
+    if (n_blocks == 0) return SPARK_OK;
+    CompressArgs A;
+    A.k = k; A.v = v; A.sb = sb; A.sh = sh; A.st = st;
+    A.lens = packed_lens; A.gather = nullptr; A.gather_stride = 0;
+    A.qnorm = qnorm; A.pages = static_cast<unsigned char*>(pages);
+    A.block_table = block_table; A.max_blocks = max_blocks; A.Hkv = p.n_kv_heads; A.keep = p.keep;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep); A.status = status;
+    const dim3 grid(n_blocks, p.n_kv_heads, p.batch);
+    if (p.dtype == SPARK_BF16)
+        compress_pages_kernel<__nv_bfloat16><<<grid, 256, A.L.page_bytes, stream>>>(A);
+    else
+        compress_pages_kernel<float><<<grid, 256, A.L.page_bytes, stream>>>(A);
+    ++*launches;
+    if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
+    return SPARK_OK;
+}
+
+spark_status launch_unpack(const spark_params& p, const void* pages, const int32_t* block_table,
+                           int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
+                           uint32_t* mask, float* mu, void* vals, void* v, cudaStream_t stream)
+{
+    const int n_blocks = (max_tokens + kPageTokens - 1) / kPageTokens;
+    if (n_blocks == 0) return SPARK_OK;
+    UnpackArgs A;
+    A.pages = static_cast<const unsigned char*>(pages); A.block_table = block_table;
+    A.max_blocks = max_blocks; A.lens = packed_lens; A.max_tokens = max_tokens; A.Hkv = p.n_kv_heads;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep);
+    A.mask = mask; A.mu = mu; A.vals = vals; A.v = v;
+    unpack_pages_kernel<<<dim3(n_blocks, p.n_kv_heads, p.batch), 128, 0, stream>>>(A);
+    if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
+    return SPARK_OK;
+}
+
+}  // namespace spark

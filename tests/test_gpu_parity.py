@@ -1,0 +1,164 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle on identical seeded inputs.
+
+Bar: kept-channel masks, kept values, value rows and qnorm bit-exact; mu within 1e-6 relative; attention
+output max|delta| <= 1e-5 (fp32 storage) / 2e-3 (bf16 storage), fp32 accumulation on the GPU.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2508_15212_b200 import binding as B
+from paper_2508_15212_b200 import build as spark_build
+from paper_2508_15212_b200 import inputs
+from paper_2508_15212_b200.cache import SparkCache
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-3}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    spark_build.build()
+    B.lib()
+
+
+def to_np(t):
+    t = t.detach().cpu()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()
+
+
+def oracle_side(wl_cpu, keep):
+    Hkv = wl_cpu.k.shape[1]
+    _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
+    c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a, want_idx=True)
+    out, lse = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a)
+    return a, c, out, lse
+
+
+def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True):
+    """wl lives on the GPU; returns max|delta| of the attention output."""
+    Bn, Hq, Hkv, W, D, S = wl.shape
+    wl_cpu = wl.to("cpu")
+    a, c, o_ref, lse_ref = oracle_side(wl_cpu, keep)
+    cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
+                       max_tokens=S, block_table=block_table, n_pool_pages=n_pool_pages)
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    lens = wl_cpu.seq_lens.tolist()
+    assert cache.packed_lens.cpu().tolist() == lens
+    assert np.array_equal(cache.qnorm.cpu().numpy(), a), "qnorm must be bit-exact"
+    u = cache.unpack()
+    mask = u["mask"].cpu().numpy().view(np.uint32)
+    assert np.array_equal(mask, c["mask"]), "kept-channel masks must be bit-exact"
+    mu = u["mu"].cpu().numpy()
+    assert np.allclose(mu, c["mu"], rtol=1e-6, atol=0)
+    if check_vals:
+        kk = to_np(wl_cpu.k)
+        want_vals = np.take_along_axis(kk, c["kept_idx"].astype(np.int64), axis=-1)
+        vv = to_np(wl_cpu.v).copy()
+        for b, n in enumerate(lens):
+            want_vals[b, :, n:] = 0
+            vv[b, :, n:] = 0
+        assert np.array_equal(to_np(u["vals"]), want_vals), "kept values must be bit-identical copies"
+        assert np.array_equal(to_np(u["v"]), vv)
+    lse = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
+    out = cache.decode(wl.q, lse=lse)
+    out2 = cache.decode(wl.q)                                    # tickets self-reset; result reproducible
+    assert cache.status() == 0
+    assert torch.equal(out, out2)
+    d = float(np.abs(out.cpu().numpy() - o_ref).max())
+    assert d <= TOL[wl.dtype], f"max|delta| {d:.3e} (max|out| {np.abs(o_ref).max():.3e})"
+    l = lse.cpu().numpy()
+    fin = np.isfinite(lse_ref)
+    assert np.array_equal(np.isneginf(l), np.isneginf(lse_ref))
+    assert np.allclose(l[fin], lse_ref[fin], rtol=0, atol=1e-3 if wl.dtype == "bf16" else 2e-5)
+    return d
+
+
+def make(dtype, Bn, Hq, Hkv, lens, W, keep, seed, sigma=1.0, gap=True):
+    wl = inputs.make_workload(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=lens, window=W, dtype=dtype,
+                              sigma_s=sigma, seed=seed, device="cuda")
+    if gap:
+        inputs.enforce_saliency_gap(wl, keep)
+    return wl
+
+
+def test_config1_tiny_fp32_full():
+    c = inputs.CONFIGS[0]
+    wl = inputs.config_workload(0, device="cuda")
+    keep = B.spark_keep_count(128, c["ratio"])
+    assert keep == 64
+    inputs.enforce_saliency_gap(wl, keep)
+    check_case(wl, keep)
+
+
+@pytest.mark.parametrize("keep", [1, 25, 26, 38, 64, 89, 127, 128])
+def test_bf16_gqa4_ragged_lengths_every_keep(keep):
+    wl = make("bf16", 3, 8, 2, [1, 37, 530], 8, keep, seed=10 + keep)
+    check_case(wl, keep)
+
+
+@pytest.mark.parametrize("G,keep", [(1, 64), (2, 38), (3, 64), (5, 25), (6, 89), (7, 64), (8, 64)])
+def test_group_sizes_bf16(G, keep):
+    wl = make("bf16", 2, 2 * G, 2, [300, 47], 16, keep, seed=40 + G)
+    check_case(wl, keep)
+
+
+@pytest.mark.parametrize("G,keep", [(1, 64), (2, 38), (4, 25), (7, 64), (8, 100)])
+def test_group_sizes_fp32(G, keep):
+    wl = make("f32", 2, 2 * G, 2, [200, 33], 8, keep, seed=60 + G, sigma=0.5)
+    check_case(wl, keep)
+
+
+def test_single_token_and_empty_sequence():
+    wl = make("bf16", 3, 8, 2, [0, 1, 16], 4, 64, seed=70)
+    check_case(wl, 64)
+
+
+def test_paged_pool_with_permuted_block_table_qwen_shape():
+    lens = [700, 33, 1200, 16]
+    wl = make("bf16", 4, 28, 4, lens, 32, 38, seed=80)
+    max_blocks = (max(lens) + 15) // 16 + 3                      # table wider than needed
+    n_pages = 4 * 4 * max_blocks + 11
+    g = torch.Generator().manual_seed(5)
+    perm = torch.randperm(n_pages, generator=g)[: 4 * 4 * max_blocks].to(torch.int32)
+    bt = perm.view(4, 4, max_blocks).cuda()
+    check_case(wl, 38, block_table=bt, n_pool_pages=n_pages)
+
+
+def test_token_major_kv_layout():
+    wl = make("bf16", 2, 8, 2, [100, 260], 8, 64, seed=90)
+    k_tm = wl.k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)      # [B,S,H,D] storage
+    v_tm = wl.v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert k_tm.stride() != wl.k.stride()
+    wl.k, wl.v = k_tm, v_tm
+    check_case(wl, 64)
+
+
+def test_many_units_cross_cta_boundaries():
+    """More (sequence, head) units than CTAs, lengths that make CTA ranges straddle units."""
+    lens = [64 + 37 * i for i in range(40)]
+    wl = make("bf16", 40, 16, 8, lens, 8, 64, seed=100, gap=False)
+    check_case(wl, 64, check_vals=False)
+
+
+def test_config2_llama_32k_full():
+    c = inputs.CONFIGS[1]
+    wl = inputs.config_workload(1, device="cuda")
+    keep = B.spark_keep_count(128, c["ratio"])
+    inputs.enforce_saliency_gap(wl, keep)
+    d = check_case(wl, keep)
+    print(f"config 2 max|delta| = {d:.3e}")
+
+
+def test_bad_page_id_is_recorded_not_dereferenced():
+    wl = make("bf16", 1, 4, 1, [64], 4, 64, seed=110, gap=False)
+    cache = SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype="bf16", max_tokens=64)
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    assert cache.status() == 0
+    cache.block_table[0, 0, 1] = 1 << 20                       # outside the pool
+    cache.decode(wl.q)
+    assert B.spark_read_status(cache.ws_decode) == 6            # SPARK_ERR_DEVICE_BOUNDS
