@@ -25,7 +25,7 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kDecodeThreads = kConsumerThreads + 32;
 constexpr int kMaxSlots = 16;
 constexpr int kStepTokens = 2 * kPageTokens;
-constexpr unsigned kSpinLimit = 1u << 22;       // bounded mbarrier waits
+constexpr unsigned kSpinLimit = 1u << 20;       // bounded mbarrier waits
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kRec = kHeadDim + 4;           // floats per (head) record: 128 accumulators, running max, running sum, pad
 
