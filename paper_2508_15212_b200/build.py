@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspark.so")
-SOURCES = ["spark_api.cu", "spark_compress.cu", "spark_decode.cu"]
-HEADERS = [os.path.join(CSRC, "spark_common.cuh"),
+SOURCES = ["spark_api.cu", "spark_compress.cu", "spark_decode.cu", "spark_decode_mma.cu"]
+HEADERS = [os.path.join(CSRC, "spark_common.cuh"), os.path.join(CSRC, "spark_decode_common.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "spark.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

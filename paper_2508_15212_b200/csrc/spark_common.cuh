@@ -19,17 +19,17 @@ constexpr int kWorkspaceHeader = 256;
 
 // Byte layout of one page (16 tokens of one KV head).  Private to the library.
 //
-//   vals : `rows` rows of 64 bytes.  bf16: row r holds slots 2r and 2r+1 of every token, token p at
-//          byte p*4 (+2 for the odd slot); fp32: row r holds slot r, token p at byte p*4.  Slot s of a
-//          token is its s-th kept channel in ascending channel order.  A row is one 64-byte line for the
-//          16 tokens, so a lane-per-token reader hits 16 distinct banks whatever slot each lane is at.
+//   vals : T rows of 16 elements.  Row s holds kept slot s of every token (token p at element p); slot s
+//          of a token is its s-th kept channel in ascending channel order.  Rows are 32 bytes (bf16) or
+//          64 bytes (fp32), so the section is exactly T elements per token.
 //   mask : [16][4] uint32, bit (j % 32) of word (j / 32) set <=> channel j kept
 //   mu   : [16] float, mean saliency of the pruned channels
-//   v    : [16][128] elements, dense value rows
+//   v    : [16][128] elements, dense value rows.  In bf16 pages the 16-byte chunks of row p are stored
+//          at chunk index (c ^ (p & 7)), which makes the transposing matrix loads of the decode kernel
+//          free of bank conflicts; fp32 pages store rows plainly.
 struct PageLayout {
     int esize;       // bytes per element (2 bf16, 4 fp32)
     int keep;        // T
-    int rows;        // ceil(T/2) for bf16, T for fp32
     int mask_off;
     int mu_off;
     int v_off;
@@ -41,8 +41,7 @@ __host__ __device__ inline PageLayout make_layout(int dtype, int keep)
     PageLayout L;
     L.esize = (dtype == SPARK_BF16) ? 2 : 4;
     L.keep = keep;
-    L.rows = (dtype == SPARK_BF16) ? (keep + 1) / 2 : keep;
-    L.mask_off = L.rows * 64;
+    L.mask_off = keep * kPageTokens * L.esize;
     L.mu_off = L.mask_off + kPageTokens * 16;
     L.v_off = L.mu_off + kPageTokens * 4;
     L.page_bytes = L.v_off + kPageTokens * kHeadDim * L.esize;
@@ -52,7 +51,13 @@ __host__ __device__ inline PageLayout make_layout(int dtype, int keep)
 // byte offset of kept slot s of token p inside the vals section
 __host__ __device__ inline int val_offset(int esize, int p, int s)
 {
-    return esize == 2 ? ((s >> 1) * 64 + p * 4 + (s & 1) * 2) : (s * 64 + p * 4);
+    return (s * kPageTokens + p) * esize;
+}
+
+// byte offset (inside the v section) of the 16-byte chunk c of token p's value row
+__host__ __device__ inline int v_chunk_offset(int esize, int p, int c)
+{
+    return esize == 2 ? (p * (kHeadDim * 2) + ((c ^ (p & 7)) << 4)) : (p * (kHeadDim * 4) + (c << 4));
 }
 
 // Workspace header: word 0 is the status word (first error wins).

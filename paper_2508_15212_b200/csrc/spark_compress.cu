@@ -105,14 +105,14 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             raw[0] = kk.x & 0xffffu; raw[1] = kk.x >> 16; raw[2] = kk.y & 0xffffu; raw[3] = kk.y >> 16;
 #pragma unroll
             for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i] << 16);
-            *reinterpret_cast<uint2*>(image + L.v_off + p * (kHeadDim * 2) + lane * 8) = vv;
+            *reinterpret_cast<uint2*>(image + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) = vv;
         } else {
             const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.k) + row);
             const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.v) + row);
             raw[0] = kk.x; raw[1] = kk.y; raw[2] = kk.z; raw[3] = kk.w;
 #pragma unroll
             for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
-            *reinterpret_cast<uint4*>(image + L.v_off + p * (kHeadDim * 4) + lane * 16) = vv;
+            *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) = vv;
         }
         float w[4];
         unsigned key[4];
@@ -252,15 +252,17 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
         }
     if (A.v)
         for (int i = threadIdx.x; i < kPageTokens * kHeadDim; i += blockDim.x) {
-            const int p = i / kHeadDim;
+            const int p = i / kHeadDim, j = i % kHeadDim;
             if (t0 + p >= A.max_tokens) continue;
             const bool live = page && t0 + p < len;
-            const int64_t o = (row0 + p) * kHeadDim + (i % kHeadDim);
-            if (L.esize == 2)
-                static_cast<unsigned short*>(A.v)[o] =
-                    live ? reinterpret_cast<const unsigned short*>(page + L.v_off)[i] : 0;
-            else
-                static_cast<unsigned*>(A.v)[o] = live ? reinterpret_cast<const unsigned*>(page + L.v_off)[i] : 0u;
+            const int64_t o = (row0 + p) * kHeadDim + j;
+            if (L.esize == 2) {
+                const unsigned char* src = page + L.v_off + v_chunk_offset(2, p, j >> 3) + (j & 7) * 2;
+                static_cast<unsigned short*>(A.v)[o] = live ? *reinterpret_cast<const unsigned short*>(src) : 0;
+            } else {
+                const unsigned char* src = page + L.v_off + v_chunk_offset(4, p, j >> 2) + (j & 3) * 4;
+                static_cast<unsigned*>(A.v)[o] = live ? *reinterpret_cast<const unsigned*>(src) : 0u;
+            }
         }
 }
 

@@ -49,9 +49,9 @@ def params(**kw):
 
 def test_page_and_algorithmic_bytes(lib):
     import torch
-    # bf16: 16 tokens * (2T + 16 + 4 + 256) bytes, T rounded up to even in storage
+    # bf16: 16 tokens * (2T + 16 + 4 + 256) bytes exactly
     assert B.spark_page_bytes(params(keep=64)) == 16 * 404
-    assert B.spark_page_bytes(params(keep=25)) == 16 * (52 + 20 + 256)
+    assert B.spark_page_bytes(params(keep=25)) == 16 * 326
     assert B.spark_page_bytes(params(keep=128)) == 16 * (256 + 20 + 256)
     assert B.spark_page_bytes(params(keep=64, dtype=torch.float32)) == 16 * 788
     assert B.spark_page_bytes(params(keep=0)) == 0 and B.spark_page_bytes(params(keep=129)) == 0
