@@ -92,11 +92,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volati
     record_error(status, SPARK_ERR_DEVICE_TIMEOUT);
     return false;
 }
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes, uint64_t* bar)
+// Bulk copy global -> shared that signals `bar`; `policy` is an L2 eviction policy (pages are read once
+// per step, so they are streamed evict-first and leave the L2 to the small tables and the partials).
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, unsigned bytes, uint64_t* bar, uint64_t policy)
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
 __device__ __forceinline__ void consumer_sync()
 {
@@ -204,6 +213,7 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
     const int max_tokens = A.max_blocks * kPageTokens;
     bool live = true;
     int issued = 0;
+    const uint64_t policy = policy_evict_first();
     for (int n0 = 0; n0 < n_total; n0 += 32) {
         const int n = n0 + lane;
         int id0 = -1, id1 = -1;
@@ -230,10 +240,10 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
                     unsigned char* dst = ring + static_cast<size_t>(slot) * A.slot_stride;
                     const unsigned bytes = L.page_bytes * (p1 >= 0 ? 2u : 1u);
                     mbar_expect_tx(&C.full[slot], bytes);
-                    bulk_g2s(dst, A.pages + static_cast<int64_t>(p0) * L.page_bytes, L.page_bytes, &C.full[slot]);
+                    bulk_g2s(dst, A.pages + static_cast<int64_t>(p0) * L.page_bytes, L.page_bytes, &C.full[slot], policy);
                     if (p1 >= 0)
                         bulk_g2s(dst + L.page_bytes, A.pages + static_cast<int64_t>(p1) * L.page_bytes,
-                                 L.page_bytes, &C.full[slot]);
+                                 L.page_bytes, &C.full[slot], policy);
                     ++issued;
                 }
             }
@@ -311,15 +321,35 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
             __threadfence();
             for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
                 const int gg = idx / kHeadDim, c = idx - gg * kHeadDim;
+                const float* r0 = A.partials + (static_cast<int64_t>(first_cta + unit) * G + gg) * kRec;
+                constexpr int kBatch = 8;                // loads of a batch are issued together
+                constexpr int64_t kStride = static_cast<int64_t>(G) * kRec;
                 float M = -INFINITY;
-                for (int pc = first_cta; pc <= last_cta; ++pc)
-                    M = fmaxf(M, __ldcg(A.partials + (static_cast<int64_t>(pc + unit) * G + gg) * kRec + kHeadDim));
+                for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
+                    float mv[kBatch];
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k)
+                        mv[k] = (p0 + k < n_parts) ? __ldcg(r0 + (p0 + k) * kStride + kHeadDim) : -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k) M = fmaxf(M, mv[k]);
+                }
                 float Ls = 0.f, O = 0.f;
-                for (int pc = first_cta; pc <= last_cta; ++pc) {
-                    const float* r = A.partials + (static_cast<int64_t>(pc + unit) * G + gg) * kRec;
-                    const float f = exp2f(__ldcg(r + kHeadDim) - M);
-                    Ls = fmaf(__ldcg(r + kHeadDim + 1), f, Ls);
-                    O = fmaf(__ldcg(r + c), f, O);
+                for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
+                    float mv[kBatch], lv[kBatch], ov[kBatch];
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k) {
+                        const bool in = p0 + k < n_parts;
+                        const float* r = r0 + (p0 + k) * kStride;
+                        mv[k] = in ? __ldcg(r + kHeadDim) : -INFINITY;
+                        lv[k] = in ? __ldcg(r + kHeadDim + 1) : 0.f;
+                        ov[k] = in ? __ldcg(r + c) : 0.f;
+                    }
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k) {
+                        const float f = exp2f(mv[k] - M);
+                        Ls = fmaf(lv[k], f, Ls);
+                        O = fmaf(ov[k], f, O);
+                    }
                 }
                 A.out[(static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + c] = O / Ls;
                 if (c == 0 && A.lse)
