@@ -43,11 +43,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
 
     decode_prologue(A, C, tid);
     const int* prefix = C.prefix;
-    const int total = A.Hkv * prefix[A.B];
-    const int nct = static_cast<int>(gridDim.x);
-    const int chunk = (total + nct - 1) / nct;
-    const int c0 = min(total, static_cast<int>(blockIdx.x) * chunk);
-    const int c1 = min(total, c0 + chunk);
+    int c0, c1;
+    cta_range(*C.plan, static_cast<int>(blockIdx.x), c0, c1);
 
     if (warp == kConsumerWarps) {
         producer_loop(A, C, ring, c0, c1, lane);
@@ -197,7 +194,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
             }
         }
         consumer_sync();
-        merge_and_publish<G>(A, C, merge, sg, chunk, tid);
+        merge_and_publish<G>(A, C, merge, sg, tid);
         g += sg.n;
         base += sg.n;
     }

@@ -147,11 +147,26 @@ __device__ __forceinline__ Segment locate(const int* prefix, int B, int Hkv, int
     return s;
 }
 
+// How the step line is divided among the CTAs.
+//   stream mode : CTA c owns steps [c*chunk, (c+1)*chunk) of the whole line; a CTA may cross unit
+//                 boundaries (exact balance; used when sequences differ in length or units are many).
+//   aligned mode: all units have the same number of steps and there are several CTAs per unit; unit u
+//                 gets q or q+1 whole CTAs (the first `rem` units get q+1) and is split evenly among
+//                 them, so no CTA crosses a unit boundary and every CTA publishes exactly once.
+struct Plan {
+    int total;        // steps on the line
+    int chunk;        // stream mode: steps per CTA
+    int aligned;      // 1: aligned mode
+    int unit_steps;   // aligned mode: steps of every unit
+    int q, rem;       // aligned mode: CTAs per unit
+};
+
 struct Ctrl {
     uint64_t* full;
     uint64_t* empty;
     volatile int* abort_flag;
     volatile int* last_flag;
+    Plan* plan;
     int* prefix;
 };
 
@@ -162,6 +177,7 @@ __device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
     c.empty = c.full + kMaxSlots;
     c.abort_flag = reinterpret_cast<volatile int*>(smem + 256);
     c.last_flag = reinterpret_cast<volatile int*>(smem + 260);
+    c.plan = reinterpret_cast<Plan*>(smem + 272);
     c.prefix = reinterpret_cast<int*>(smem + kCtrlBytes);
     return c;
 }
@@ -179,7 +195,7 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 0) {
-        int running = 0;
+        int running = 0, smin = 0x7fffffff, smax = 0;
         for (int b0 = 0; b0 < A.B; b0 += 32) {
             const int b = b0 + lane;
             int st = 0;
@@ -187,6 +203,8 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
                 const int len = A.lens[b];
                 if (len < 0 || len > max_tokens) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
                 st = steps_of(clamp_len(len, max_tokens));
+                smin = min(smin, st);
+                smax = max(smax, st);
             }
             int inc = st;
 #pragma unroll
@@ -197,9 +215,61 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
             if (b < A.B) C.prefix[b + 1] = running + inc;
             running += __shfl_sync(kFull, inc, 31);
         }
-        if (lane == 0) C.prefix[0] = 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            smin = min(smin, __shfl_xor_sync(kFull, smin, o));
+            smax = max(smax, __shfl_xor_sync(kFull, smax, o));
+        }
+        if (lane == 0) {
+            C.prefix[0] = 0;
+            Plan pl;
+            const int nct = static_cast<int>(gridDim.x), units = A.B * A.Hkv;
+            pl.total = A.Hkv * running;
+            pl.chunk = (pl.total + nct - 1) / nct;
+            pl.aligned = 0; pl.unit_steps = smax; pl.q = 0; pl.rem = 0;
+            if (smin == smax && smax > 0 && units <= nct) {
+                const int q = nct / units;
+                const int makespan = (smax + q - 1) / q;
+                if (q >= 2 && makespan * 25 <= pl.chunk * 26) {          // within 4 % of the even split
+                    pl.aligned = 1; pl.q = q; pl.rem = nct - q * units;
+                }
+            }
+            *C.plan = pl;
+        }
     }
     __syncthreads();
+}
+
+// This CTA's run of steps [c0, c1) on the line.
+__device__ __forceinline__ void cta_range(const Plan& pl, int cta, int& c0, int& c1)
+{
+    if (!pl.aligned) {
+        c0 = min(pl.total, cta * pl.chunk);
+        c1 = min(pl.total, c0 + pl.chunk);
+        return;
+    }
+    const int big = pl.rem * (pl.q + 1);                   // CTAs that belong to units with q+1 CTAs
+    int u, k, n;
+    if (cta < big) { u = cta / (pl.q + 1); k = cta - u * (pl.q + 1); n = pl.q + 1; }
+    else { u = pl.rem + (cta - big) / pl.q; k = (cta - big) - (u - pl.rem) * pl.q; n = pl.q; }
+    const int per = (pl.unit_steps + n - 1) / n;
+    c0 = u * pl.unit_steps + min(pl.unit_steps, k * per);
+    c1 = u * pl.unit_steps + min(pl.unit_steps, (k + 1) * per);
+}
+
+// The CTAs that hold a part of the unit starting at step `unit_start` with `unit_steps` steps.
+__device__ __forceinline__ void unit_parts(const Plan& pl, int unit_start, int unit_steps, int& first_cta, int& n_parts)
+{
+    if (!pl.aligned) {
+        first_cta = unit_start / pl.chunk;
+        n_parts = (unit_start + unit_steps - 1) / pl.chunk - first_cta + 1;
+        return;
+    }
+    const int u = unit_start / pl.unit_steps;
+    const int n = pl.q + (u < pl.rem ? 1 : 0);
+    first_cta = u * pl.q + min(u, pl.rem);
+    const int per = (pl.unit_steps + n - 1) / n;
+    n_parts = (pl.unit_steps + per - 1) / per;             // trailing CTAs of the unit may be empty
 }
 
 // The producer warp: walks this CTA's steps [c0, c1) in order, looks the page ids up 32 steps at a
@@ -279,12 +349,11 @@ __device__ __forceinline__ void write_empty_sequences(const DecodeArgs& A, const
 // consumer threads after a consumer_sync(); ends with a consumer_sync().
 template <int G>
 __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctrl& C, const float* merge,
-                                                  const Segment& sg, int chunk, int tid)
+                                                  const Segment& sg, int tid)
 {
     const int b = sg.b, h = sg.h;
-    const int unit_end = sg.unit_start + sg.steps_b;
-    const int first_cta = sg.unit_start / chunk, last_cta = (unit_end - 1) / chunk;
-    const int n_parts = last_cta - first_cta + 1;
+    int first_cta, n_parts;
+    unit_parts(*C.plan, sg.unit_start, sg.steps_b, first_cta, n_parts);
     const int unit = b * A.Hkv + h;
     float* part_out = A.partials + static_cast<int64_t>(blockIdx.x + unit) * G * kRec;
     for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
@@ -310,30 +379,23 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
         }
     }
     if (n_parts > 1) {
-        __threadfence();
+        // The barrier orders every consumer thread's partial stores before thread 0's gpu-scope
+        // release; the last arriver's acquire (same atomic) plus the next barrier orders its reads
+        // after all partials.
         consumer_sync();
         if (tid == 0) {
-            const int old = atomicAdd(&A.tickets[unit], 1);
+            int old;
+            asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(A.tickets + unit) : "memory");
             *C.last_flag = (old == n_parts - 1) ? 1 : 0;
         }
         consumer_sync();
         if (*C.last_flag) {                              // last CTA of this unit: merge all partials
-            __threadfence();
+            constexpr int kBatch = 20;                   // loads of a batch are in flight together
+            constexpr int64_t kStride = static_cast<int64_t>(G) * kRec;
             for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
                 const int gg = idx / kHeadDim, c = idx - gg * kHeadDim;
                 const float* r0 = A.partials + (static_cast<int64_t>(first_cta + unit) * G + gg) * kRec;
-                constexpr int kBatch = 8;                // loads of a batch are issued together
-                constexpr int64_t kStride = static_cast<int64_t>(G) * kRec;
-                float M = -INFINITY;
-                for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
-                    float mv[kBatch];
-#pragma unroll
-                    for (int k = 0; k < kBatch; ++k)
-                        mv[k] = (p0 + k < n_parts) ? __ldcg(r0 + (p0 + k) * kStride + kHeadDim) : -INFINITY;
-#pragma unroll
-                    for (int k = 0; k < kBatch; ++k) M = fmaxf(M, mv[k]);
-                }
-                float Ls = 0.f, O = 0.f;
+                float M = -INFINITY, Ls = 0.f, O = 0.f;
                 for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
                     float mv[kBatch], lv[kBatch], ov[kBatch];
 #pragma unroll
@@ -344,12 +406,19 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
                         lv[k] = in ? __ldcg(r + kHeadDim + 1) : 0.f;
                         ov[k] = in ? __ldcg(r + c) : 0.f;
                     }
+                    float Mn = M;
+#pragma unroll
+                    for (int k = 0; k < kBatch; ++k) Mn = fmaxf(Mn, mv[k]);
+                    const float sc = exp2f(M - Mn);      // 0 for the first batch
+                    Ls *= sc;
+                    O *= sc;
 #pragma unroll
                     for (int k = 0; k < kBatch; ++k) {
-                        const float f = exp2f(mv[k] - M);
+                        const float f = exp2f(mv[k] - Mn);
                         Ls = fmaf(lv[k], f, Ls);
                         O = fmaf(ov[k], f, O);
                     }
+                    M = Mn;
                 }
                 A.out[(static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + c] = O / Ls;
                 if (c == 0 && A.lse)

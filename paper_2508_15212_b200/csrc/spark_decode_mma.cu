@@ -136,11 +136,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const De
 
     decode_prologue(A, C, tid);
     const int* prefix = C.prefix;
-    const int total = A.Hkv * prefix[A.B];
-    const int nct = static_cast<int>(gridDim.x);
-    const int chunk = (total + nct - 1) / nct;
-    const int c0 = min(total, static_cast<int>(blockIdx.x) * chunk);
-    const int c1 = min(total, c0 + chunk);
+    int c0, c1;
+    cta_range(*C.plan, static_cast<int>(blockIdx.x), c0, c1);
 
 #ifdef SPARK_CTA_TIMING
     unsigned long long t_start = 0, t_first = 0, t_probe[12];
@@ -337,7 +334,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const De
         }
         consumer_sync();
         SPARK_PROBE();      // all warps done
-        merge_and_publish<G>(A, C, merge, sg, chunk, tid);
+        merge_and_publish<G>(A, C, merge, sg, tid);
         SPARK_PROBE();      // published
         g += sg.n;
         base += sg.n;
