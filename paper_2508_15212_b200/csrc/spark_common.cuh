@@ -14,7 +14,7 @@ constexpr int kPageTokens = 16;      // P
 constexpr int kMaskWords = 4;        // 128-bit channel mask per token
 constexpr int kMaxGroup = 8;         // G = Hq / Hkv
 constexpr int kMaxBatch = 1024;      // sequences per call (decode keeps a per-sequence prefix in shared memory)
-constexpr int kMaxCtas = 1024;       // upper bound of the persistent decode grid (sizes the partial-result slots)
+constexpr int kMaxCtas = 256;        // upper bound of the persistent decode grid (sizes the partial-result slots)
 constexpr int kWorkspaceHeader = 256;
 
 // Byte layout of one page (16 tokens of one KV head).  Private to the library.

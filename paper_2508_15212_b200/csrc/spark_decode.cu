@@ -13,6 +13,11 @@
 
 namespace spark {
 
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kDecodeThreads = kConsumerThreads + 32;     // + producer warp
+constexpr int kStepTokens = 2 * kPageTokens;              // a lane per token: two pages per step
+
 template <int G> struct SmemF32 {
     static constexpr int GP = ((G + 1 + 3) / 4) * 4;     // floats per table entry: G scaled queries + 1/a
     static constexpr int GPP = ((G + 3) / 4) * 4;        // floats per probability entry
@@ -20,7 +25,7 @@ template <int G> struct SmemF32 {
     static constexpr int kQsum = kQtab + kHeadDim * GP * 4;
     static constexpr int kPscr = kQsum + 32;
     static constexpr int kMerge = kPscr + kConsumerWarps * 32 * GPP * 4;
-    static constexpr int kRing = (kMerge + kConsumerWarps * G * kRec * 4 + 127) / 128 * 128;
+    static constexpr int kRing = (kMerge + merge_bytes(kConsumerWarps, G) + 127) / 128 * 128;
 };
 
 template <int G>
@@ -50,7 +55,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
         producer_loop(A, C, ring, c0, c1, lane);
         return;
     }
-    write_empty_sequences(A, prefix, tid);
+    write_empty_sequences<kConsumerThreads>(A, prefix, tid);
 
     float* pscr = pscr_all + warp * 32 * GPP;
     int base = 0;                                          // ordinal (within this CTA) of the segment's first step
@@ -70,7 +75,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                 val = 1.0f / A.qnorm[(static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + j];
             qtab[idx] = val;
         }
-        consumer_sync();
+        consumer_sync<kConsumerThreads>();
         if (warp < G) {                                    // Qsum[g] = sum_j q_g[j]*c / a[j]
             double part = 0.0;
 #pragma unroll
@@ -82,7 +87,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
             for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFull, part, o);
             if (lane == 0) qsum[warp] = static_cast<float>(part);
         }
-        consumer_sync();
+        consumer_sync<kConsumerThreads>();
 
         float m_run[G], l_run[G], acc[G][4];
 #pragma unroll
@@ -193,8 +198,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                 mine[gg * kRec + kHeadDim + 1] = lsum;
             }
         }
-        consumer_sync();
-        merge_and_publish<G>(A, C, merge, sg, tid);
+        consumer_sync<kConsumerThreads>();
+        merge_and_publish<G, kConsumerWarps>(A, C, merge, sg, tid);
         g += sg.n;
         base += sg.n;
     }
@@ -218,6 +223,7 @@ static spark_status launch_f32(const DecodeArgs& A0, int n_sms, int smem_optin, 
 {
     DecodeArgs A = A0;
     using S = SmemF32<G>;
+    A.pps = 2;
     A.slot_stride = static_cast<int>(align_up(2 * static_cast<size_t>(A.L.page_bytes), 128));
     int ns = (smem_optin - S::kRing) / A.slot_stride;
     if (ns > kMaxSlots) ns = kMaxSlots;
@@ -271,7 +277,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.status = reinterpret_cast<int*>(ws);
     A.tickets = reinterpret_cast<int*>(ws + kWorkspaceHeader);
     A.partials = reinterpret_cast<float*>(ws + kWorkspaceHeader + align_up(units * sizeof(int), 256));
-    A.nslots = 0; A.slot_stride = 0;
+    A.nslots = 0; A.slot_stride = 0; A.pps = 1;
     const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, n_sms, smem_optin, stream)
                                                     : launch_decode_f32(G, A, n_sms, smem_optin, stream);
     if (st == SPARK_OK) ++*launches;

@@ -1,25 +1,20 @@
 // Pieces shared by the decode kernels: launch arguments, mbarrier / bulk-copy PTX wrappers, the
 // division of the step line among CTAs, the producer warp, and the merge of partial softmax states.
 //
-// Execution shape (both kernels): a persistent grid of one CTA per SM.  The (sequence, KV head) units
-// are cut into steps of two pages (32 tokens); the steps of all units form one line that is divided
-// evenly among the CTAs, so a CTA owns a contiguous run of steps that may cross unit boundaries.
-// Inside a CTA one producer warp streams pages into a shared-memory ring with bulk asynchronous copies
-// that signal mbarriers; eight consumer warps each take whole steps and keep an online-softmax state
-// (running max m in the log2 domain, running sum l, unnormalised output).  At the end of a unit's run
-// the warps are merged by log-sum-exp; if several CTAs share the unit each writes a partial and the
-// last to arrive (an atomic ticket, no waiting) merges them.
+// Execution shape (both kernels): a persistent grid of one CTA per SM.  Every (sequence, KV head) unit
+// is cut into steps of `pps` pages (16 or 32 tokens); the steps of all units form one line that is
+// divided among the CTAs.  Inside a CTA one producer warp streams pages into a shared-memory ring with
+// bulk asynchronous copies that signal mbarriers; NW consumer warps each take whole steps and keep an
+// online-softmax state (running max m in the log2 domain, running sum l, unnormalised output).  At
+// the end of a unit's run the warps are merged by log-sum-exp; if several CTAs share the unit each
+// writes a partial and the last to arrive (an atomic ticket, no waiting) merges them.
 #pragma once
 
 #include "spark_common.cuh"
 
 namespace spark {
 
-constexpr int kConsumerWarps = 8;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kDecodeThreads = kConsumerThreads + 32;
-constexpr int kMaxSlots = 16;
-constexpr int kStepTokens = 2 * kPageTokens;
+constexpr int kMaxSlots = 32;
 constexpr unsigned kSpinLimit = 1u << 20;    // bounded mbarrier waits
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kRec = kHeadDim + 4;           // floats per head record: 128 outputs, running max, running sum, pad
@@ -43,11 +38,20 @@ struct DecodeArgs {
     float* partials;
     int nslots;
     int slot_stride;
+    int pps;                                 // pages per step (= per ring slot): 1 or 2
 };
 
 // control block at the start of dynamic shared memory
-constexpr int kCtrlBytes = 512;                                  // full[16], empty[16], flags
+constexpr int kCtrlBytes = 1024;                                 // full[32], empty[32], flags, plan
 constexpr int kPrefixBytes = ((kMaxBatch + 1) * 4 + 15) / 16 * 16;
+
+// Bytes of the shared merge area for `nw` consumer warps and `g` heads.  The final combine reuses it
+// for the (m, l) pairs of up to kMaxCtas parts followed by one float4 per consumer thread.
+__host__ __device__ constexpr int merge_bytes(int nw, int g)
+{
+    return nw * g * kRec * 4 > kMaxCtas * g * 8 + nw * 32 * 16 ? nw * g * kRec * 4
+                                                               : kMaxCtas * g * 8 + nw * 32 * 16;
+}
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void* p)
@@ -107,14 +111,14 @@ __device__ __forceinline__ uint64_t policy_evict_first()
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
-__device__ __forceinline__ void consumer_sync()
+template <int NT> __device__ __forceinline__ void consumer_sync()
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
 }
 
-__device__ __forceinline__ int steps_of(int len)
+__device__ __forceinline__ int steps_of(int len, int pps)
 {
-    return ((len + kPageTokens - 1) / kPageTokens + 1) >> 1;
+    return ((len + kPageTokens - 1) / kPageTokens + pps - 1) / pps;
 }
 
 __device__ __forceinline__ int clamp_len(int len, int max_tokens)
@@ -175,19 +179,20 @@ __device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
     Ctrl c;
     c.full = reinterpret_cast<uint64_t*>(smem);
     c.empty = c.full + kMaxSlots;
-    c.abort_flag = reinterpret_cast<volatile int*>(smem + 256);
-    c.last_flag = reinterpret_cast<volatile int*>(smem + 260);
-    c.plan = reinterpret_cast<Plan*>(smem + 272);
+    c.abort_flag = reinterpret_cast<volatile int*>(smem + 512);
+    c.last_flag = reinterpret_cast<volatile int*>(smem + 516);
+    c.plan = reinterpret_cast<Plan*>(smem + 528);
     c.prefix = reinterpret_cast<int*>(smem + kCtrlBytes);
     return c;
 }
 
-// Barrier init (thread 0) and the steps-per-sequence prefix (warp 0).  Ends with __syncthreads().
+// Barrier init (one thread of warp 1), the steps-per-sequence prefix and the plan (warp 0).
+// Ends with __syncthreads().
 __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl& C, int tid)
 {
     const int warp = tid >> 5, lane = tid & 31;
     const int max_tokens = A.max_blocks * kPageTokens;
-    if (tid == 0) {
+    if (tid == 32) {
         for (int s = 0; s < A.nslots; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], 1); }
         *C.abort_flag = 0;
         *C.last_flag = 0;
@@ -202,7 +207,7 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
             if (b < A.B) {
                 const int len = A.lens[b];
                 if (len < 0 || len > max_tokens) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
-                st = steps_of(clamp_len(len, max_tokens));
+                st = steps_of(clamp_len(len, max_tokens), A.pps);
                 smin = min(smin, st);
                 smax = max(smax, st);
             }
@@ -272,98 +277,110 @@ __device__ __forceinline__ void unit_parts(const Plan& pl, int unit_start, int u
     n_parts = (pl.unit_steps + per - 1) / per;             // trailing CTAs of the unit may be empty
 }
 
-// The producer warp: walks this CTA's steps [c0, c1) in order, looks the page ids up 32 steps at a
-// time, and lane 0 issues one or two page copies per step into ring slot (ordinal % nslots) once the
-// consumers have released it.
+// The producer warp.  Lane i owns ring slot i: it handles this CTA's steps i, i + nslots, i + 2 nslots,
+// ... in order.  Per revolution of the ring every lane looks up the page ids of its step (block-table
+// loads of the next revolution are issued before the current one is polled, so their latency hides
+// behind the wait), then the warp polls: a lane whose slot has been released by the consumers arms
+// the slot's barrier and issues its page copies at once.  Polling is bounded; on expiry the CTA-wide
+// abort flag is set and the lanes wait (bounded) for their own copies in flight before returning.
+__device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctrl& C, int g, int c1, bool active,
+                                                  int& id0, int& id1)
+{
+    id0 = -1; id1 = -1;
+    if (!active) return;
+    const int max_tokens = A.max_blocks * kPageTokens;
+    const Segment s = locate(C.prefix, A.B, A.Hkv, g, c1);
+    const int len = clamp_len(A.lens[s.b], max_tokens);
+    const int nblk = (len + kPageTokens - 1) / kPageTokens;
+    const int32_t* bt = A.block_table + (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
+    id0 = bt[A.pps * s.i0];
+    if (A.pps == 2 && 2 * s.i0 + 1 < nblk) {
+        id1 = bt[2 * s.i0 + 1];
+        if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
+    }
+    if (id0 < 0 || id0 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id0 = 0; }
+}
+
 __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C, unsigned char* ring,
                                               int c0, int c1, int lane)
 {
     const PageLayout L = A.L;
     const int NS = A.nslots, n_total = c1 - c0;
-    const int max_tokens = A.max_blocks * kPageTokens;
-    bool live = true;
-    int issued = 0;
     const uint64_t policy = policy_evict_first();
-    for (int n0 = 0; n0 < n_total; n0 += 32) {
-        const int n = n0 + lane;
-        int id0 = -1, id1 = -1;
-        if (n < n_total) {
-            const Segment s = locate(C.prefix, A.B, A.Hkv, c0 + n, c1);
-            const int len = clamp_len(A.lens[s.b], max_tokens);
-            const int nblk = (len + kPageTokens - 1) / kPageTokens;
-            const int32_t* bt = A.block_table + (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
-            id0 = bt[2 * s.i0];
-            if (2 * s.i0 + 1 < nblk) {
-                id1 = bt[2 * s.i0 + 1];
-                if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
+    const bool owner = lane < NS;
+    unsigned char* dst = ring + static_cast<size_t>(lane) * A.slot_stride;
+    uint64_t* full = &C.full[owner ? lane : 0];
+    uint64_t* empty = &C.empty[owner ? lane : 0];
+    bool live = true;
+    int last_round = -1;                                   // last revolution in which this lane issued
+    int id0, id1;
+    producer_page_ids(A, C, c0 + lane, c1, owner && lane < n_total, id0, id1);
+    for (int round = 0; round * NS < n_total; ++round) {
+        const int n = round * NS + lane;
+        bool pending = owner && n < n_total;
+        const int cur0 = id0, cur1 = id1;
+        // next revolution's ids: loads in flight while this revolution is polled
+        producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
+        unsigned it = 0;
+        while (__any_sync(kFull, pending)) {
+            if (pending && (round == 0 || mbar_try_wait(empty, (round - 1) & 1))) {
+                const unsigned bytes = L.page_bytes * (cur1 >= 0 ? 2u : 1u);
+                mbar_expect_tx(full, bytes);
+                bulk_g2s(dst, A.pages + static_cast<int64_t>(cur0) * L.page_bytes, L.page_bytes, full, policy);
+                if (cur1 >= 0)
+                    bulk_g2s(dst + L.page_bytes, A.pages + static_cast<int64_t>(cur1) * L.page_bytes,
+                             L.page_bytes, full, policy);
+                last_round = round;
+                pending = false;
             }
-            if (id0 < 0 || id0 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id0 = 0; }
+            if (++it >= kSpinLimit || *C.abort_flag) { live = false; break; }
         }
-        const int cnt = min(32, n_total - n0);
-        for (int kk = 0; kk < cnt; ++kk) {
-            const int p0 = __shfl_sync(kFull, id0, kk);
-            const int p1 = __shfl_sync(kFull, id1, kk);
-            if (lane == 0 && live) {
-                const int nn = n0 + kk, slot = nn % NS, round = nn / NS;
-                if (round > 0) live = mbar_wait(&C.empty[slot], (round - 1) & 1, C.abort_flag, A.status);
-                if (live) {
-                    unsigned char* dst = ring + static_cast<size_t>(slot) * A.slot_stride;
-                    const unsigned bytes = L.page_bytes * (p1 >= 0 ? 2u : 1u);
-                    mbar_expect_tx(&C.full[slot], bytes);
-                    bulk_g2s(dst, A.pages + static_cast<int64_t>(p0) * L.page_bytes, L.page_bytes, &C.full[slot], policy);
-                    if (p1 >= 0)
-                        bulk_g2s(dst + L.page_bytes, A.pages + static_cast<int64_t>(p1) * L.page_bytes,
-                                 L.page_bytes, &C.full[slot], policy);
-                    ++issued;
-                }
-            }
-        }
+        if (!live) break;
     }
-    // after a give-up: let the copies already in flight land before the CTA may exit
-    if (lane == 0 && !live) {
-        for (int nn = max(0, issued - NS); nn < issued; ++nn) {
-            uint64_t* bar = &C.full[nn % NS];
-            const unsigned parity = (nn / NS) & 1;
+    if (!live) {
+        if (lane == 0) { *C.abort_flag = 1; record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT); }
+        if (last_round >= 0)                               // let this lane's copy in flight land
             for (unsigned it = 0; it < kSpinLimit; ++it)
-                if (mbar_try_wait(bar, parity)) break;
-        }
+                if (mbar_try_wait(full, last_round & 1)) break;
     }
 }
 
 // zero-length sequences: out = 0, lse = -inf (consumer threads)
+template <int NT>
 __device__ __forceinline__ void write_empty_sequences(const DecodeArgs& A, const int* prefix, int tid)
 {
     for (int b = blockIdx.x; b < A.B; b += gridDim.x)
         if (prefix[b + 1] == prefix[b]) {
-            for (int i = tid; i < A.Hq * kHeadDim; i += kConsumerThreads)
+            for (int i = tid; i < A.Hq * kHeadDim; i += NT)
                 A.out[static_cast<int64_t>(b) * A.Hq * kHeadDim + i] = 0.f;
             if (A.lse)
-                for (int i = tid; i < A.Hq; i += kConsumerThreads)
+                for (int i = tid; i < A.Hq; i += NT)
                     A.lse[static_cast<int64_t>(b) * A.Hq + i] = -INFINITY;
         }
 }
 
-// Merge the per-warp states that the consumer warps have written to `merge`
+// Merge the per-warp states that the NW consumer warps have written to `merge`
 // ([warp][G][kRec]: 128 unnormalised outputs, m, l) and publish the unit's result: directly when this
 // CTA covers the whole unit, else as a partial followed by the last-arriver merge.  Called by all
 // consumer threads after a consumer_sync(); ends with a consumer_sync().
-template <int G>
-__device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctrl& C, const float* merge,
+template <int G, int NW>
+__device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctrl& C, float* merge,
                                                   const Segment& sg, int tid)
 {
+    constexpr int NT = NW * 32;
     const int b = sg.b, h = sg.h;
     int first_cta, n_parts;
     unit_parts(*C.plan, sg.unit_start, sg.steps_b, first_cta, n_parts);
     const int unit = b * A.Hkv + h;
     float* part_out = A.partials + static_cast<int64_t>(blockIdx.x + unit) * G * kRec;
-    for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
+    for (int idx = tid; idx < G * kHeadDim; idx += NT) {
         const int gg = idx / kHeadDim, c = idx - gg * kHeadDim;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge[(w * G + gg) * kRec + kHeadDim]);
+        for (int w = 0; w < NW; ++w) M = fmaxf(M, merge[(w * G + gg) * kRec + kHeadDim]);
         float Ls = 0.f, O = 0.f;
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
+        for (int w = 0; w < NW; ++w) {
             const float* r = merge + (w * G + gg) * kRec;
             const float f = exp2f(r[kHeadDim] - M);
             Ls = fmaf(r[kHeadDim + 1], f, Ls);
@@ -382,52 +399,84 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
         // The barrier orders every consumer thread's partial stores before thread 0's gpu-scope
         // release; the last arriver's acquire (same atomic) plus the next barrier orders its reads
         // after all partials.
-        consumer_sync();
+        consumer_sync<NT>();
         if (tid == 0) {
             int old;
             asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(A.tickets + unit) : "memory");
             *C.last_flag = (old == n_parts - 1) ? 1 : 0;
         }
-        consumer_sync();
-        if (*C.last_flag) {                              // last CTA of this unit: merge all partials
-            constexpr int kBatch = 20;                   // loads of a batch are in flight together
+        consumer_sync<NT>();
+        if (*C.last_flag) {
+            // Last CTA of this unit: merge all partials.  Every load is issued before the first use:
+            // thread (ph, g, c4) fetches channels 4*c4..4*c4+3 of head g for parts ph, ph+PH, ...
+            // while the (m, l) pairs of all parts go to shared memory; after one barrier the weights
+            // are known, and the weighted sums are reduced over ph through shared memory.
+            constexpr int TPG = G * 32;                  // threads per part group
+            constexpr int PH = NT / TPG;                 // part groups
+            constexpr int kBatch = 16;
             constexpr int64_t kStride = static_cast<int64_t>(G) * kRec;
-            for (int idx = tid; idx < G * kHeadDim; idx += kConsumerThreads) {
-                const int gg = idx / kHeadDim, c = idx - gg * kHeadDim;
-                const float* r0 = A.partials + (static_cast<int64_t>(first_cta + unit) * G + gg) * kRec;
-                float M = -INFINITY, Ls = 0.f, O = 0.f;
-                for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
-                    float mv[kBatch], lv[kBatch], ov[kBatch];
+            float* ml = merge;                           // [n_parts][G][2], n_parts <= kMaxCtas
+            float4* red = reinterpret_cast<float4*>(merge + kMaxCtas * G * 2);
+            const float* base = A.partials + static_cast<int64_t>(first_cta + unit) * G * kRec;
+            const int ph = tid / TPG, rem = tid - ph * TPG, gg = rem >> 5, c4 = rem & 31;
+            const bool worker = ph < PH;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float M = -INFINITY;
+            for (int p0 = 0; p0 < n_parts; p0 += kBatch * PH) {
+                float4 o4[kBatch];
 #pragma unroll
-                    for (int k = 0; k < kBatch; ++k) {
-                        const bool in = p0 + k < n_parts;
-                        const float* r = r0 + (p0 + k) * kStride;
-                        mv[k] = in ? __ldcg(r + kHeadDim) : -INFINITY;
-                        lv[k] = in ? __ldcg(r + kHeadDim + 1) : 0.f;
-                        ov[k] = in ? __ldcg(r + c) : 0.f;
-                    }
-                    float Mn = M;
-#pragma unroll
-                    for (int k = 0; k < kBatch; ++k) Mn = fmaxf(Mn, mv[k]);
-                    const float sc = exp2f(M - Mn);      // 0 for the first batch
-                    Ls *= sc;
-                    O *= sc;
-#pragma unroll
-                    for (int k = 0; k < kBatch; ++k) {
-                        const float f = exp2f(mv[k] - Mn);
-                        Ls = fmaf(lv[k], f, Ls);
-                        O = fmaf(ov[k], f, O);
-                    }
-                    M = Mn;
+                for (int k = 0; k < kBatch; ++k) {
+                    const int p = p0 + k * PH + ph;
+                    o4[k] = (worker && p < n_parts)
+                                ? *reinterpret_cast<const float4*>(base + p * kStride + gg * kRec + 4 * c4)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-                A.out[(static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + c] = O / Ls;
-                if (c == 0 && A.lse)
+                if (p0 == 0) {
+                    for (int i = tid; i < n_parts * G; i += NT) {
+                        const int p = i / G, g2 = i - p * G;
+                        const float2 v = *reinterpret_cast<const float2*>(base + p * kStride + g2 * kRec + kHeadDim);
+                        ml[2 * i] = v.x;
+                        ml[2 * i + 1] = v.y;
+                    }
+                    consumer_sync<NT>();
+                    if (worker)
+                        for (int p = 0; p < n_parts; ++p) M = fmaxf(M, ml[2 * (p * G + gg)]);
+                }
+#pragma unroll
+                for (int k = 0; k < kBatch; ++k) {
+                    const int p = p0 + k * PH + ph;
+                    if (worker && p < n_parts) {
+                        const float f = exp2f(ml[2 * (p * G + gg)] - M);
+                        acc.x = fmaf(o4[k].x, f, acc.x); acc.y = fmaf(o4[k].y, f, acc.y);
+                        acc.z = fmaf(o4[k].z, f, acc.z); acc.w = fmaf(o4[k].w, f, acc.w);
+                    }
+                }
+            }
+            float Ls = 0.f;
+            if (worker)
+                for (int p = 0; p < n_parts; ++p)
+                    Ls = fmaf(ml[2 * (p * G + gg) + 1], exp2f(ml[2 * (p * G + gg)] - M), Ls);
+            if (PH > 1) {
+                if (worker && ph > 0) red[tid] = acc;
+                consumer_sync<NT>();
+                if (ph == 0)
+#pragma unroll
+                    for (int k = 1; k < PH; ++k) {
+                        const float4 v = red[k * TPG + tid];
+                        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    }
+            }
+            if (ph == 0) {
+                const float inv = 1.0f / Ls;
+                *reinterpret_cast<float4*>(A.out + (static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + 4 * c4) =
+                    make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                if (c4 == 0 && A.lse)
                     A.lse[static_cast<int64_t>(b) * A.Hq + h * G + gg] = (M + log2f(Ls)) * kLn2;
             }
             if (tid == 0) A.tickets[unit] = 0;          // ready for the next call
         }
     }
-    consumer_sync();
+    consumer_sync<NT>();
 }
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -3,28 +3,35 @@
 //
 // For one query head, with a[j] = max(|q-bar_j|, eps) and q'[j] = q[j] / a[j]:
 //     q . K~[t] = sum_{j kept} q[j] K[t][j]  +  mu[t] * ( sum_j q'[j]  -  sum_{j kept} q'[j] ).
-// Both kept-channel sums are contractions over the 128 channels of [heads x channels] by
-// [channels x tokens], so they run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 out):
-//   - first operand rows: the G query heads (bf16, exact) for the first sum; q' split into a bf16 high
-//     and low part (rows r and r+8) for the second;
-//   - second operand: the token's kept values expanded to dense form for the first sum, and the
-//     token's mask as 0/1 for the second.  The expansion happens in registers: the four lanes that
-//     hold a token's column each own one 32-bit mask word, walk its eight nibbles, and pull the next
-//     kept value from shared memory for every set bit.  The channel order inside a k-step is a fixed
-//     permutation (lane c, step s  <->  channels 32c+4s .. 32c+4s+3) applied to both operands.
-// P.V is the third contraction: probabilities (bf16 high and low parts in rows r and r+8, so the
-// product keeps ~16 mantissa bits) by value rows fetched with transposing matrix loads; the value rows
-// are stored chunk-swizzled in the page so those loads are conflict free.  Softmax statistics and all
-// accumulators are fp32.
+// Both kept-channel sums are contractions over the 128 channels, [tokens x channels] by
+// [channels x heads], so they run on the tensor cores (mma.sync m16n8k16, bf16 in, fp32 out) with the
+// 16 tokens of a page as the rows:
+//   - first operand: the tokens' kept values expanded to dense form (first sum) and the tokens' masks
+//     as 0/1 (second sum).  The expansion happens in registers: the four lanes that hold a token row
+//     each own one 32-bit mask word, walk its eight nibbles, and pull the next kept value from shared
+//     memory for every set bit (predicated loads).  The channel order inside a k-step is a fixed
+//     permutation (lane c, step s  <->  channels 32c+4s .. 32c+4s+3) applied to both operands;
+//   - second operand (constant per unit, kept in registers): the G query heads as stored (bf16) for
+//     the first sum, and q' split into a bf16 high and low part for the second.  With G <= 4 the high
+//     and low parts share one 8-column operand (columns 0-3 / 4-7); otherwise they are two operands.
+// P.V is the third contraction, [channels x tokens] by [tokens x heads]: value rows come in through
+// transposing matrix loads (the rows are stored chunk-swizzled in the page, so these are conflict
+// free) and the probabilities, split in bf16 high and low parts so the product keeps ~16 mantissa
+// bits, are moved from the score layout to the operand layout with a warp matrix transpose.
+// Softmax statistics and all accumulators are fp32.
 #include "spark_decode_common.cuh"
 
 namespace spark {
+
+constexpr int kNW = 15;                       // consumer warps (+ 1 producer warp = 16 warps, 4 per scheduler)
+constexpr int kNT = kNW * 32;
+constexpr int kThreads = kNT + 32;
 
 template <int G> struct SmemBf16 {
     static constexpr int kTab = kCtrlBytes + kPrefixBytes;                       // q, q' high, q' low: 3 x [G][128] bf16
     static constexpr int kQsum = kTab + 3 * G * kHeadDim * 2;                    // [8] float
     static constexpr int kMerge = kQsum + 32;
-    static constexpr int kRing = (kMerge + kConsumerWarps * G * kRec * 4 + 127) / 128 * 128;
+    static constexpr int kRing = (kMerge + merge_bytes(kNW, G) + 127) / 128 * 128;
 };
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -36,11 +43,20 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ void ldmatrix_x4_trans(unsigned (&r)[4], unsigned smem_addr)
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, unsigned smem_addr)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                  : "r"(smem_addr));
+}
+
+// 8x8 b16 transpose across the warp: lane (r, c) gives row r, columns 2c..2c+1 and receives
+// rows 2c..2c+1 of column r.
+__device__ __forceinline__ unsigned movmatrix_trans(unsigned x)
+{
+    unsigned y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
 }
 
 __device__ __forceinline__ unsigned lds_u32(unsigned addr)
@@ -49,10 +65,10 @@ __device__ __forceinline__ unsigned lds_u32(unsigned addr)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ float2 lds_f32x2(unsigned addr)
+__device__ __forceinline__ float lds_f32(unsigned addr)
 {
-    float2 v;
-    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint4 lds_u32x4(unsigned addr)
@@ -60,6 +76,12 @@ __device__ __forceinline__ uint4 lds_u32x4(unsigned addr)
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ unsigned pack_bf16(float lo, float hi)
@@ -73,7 +95,7 @@ __device__ __forceinline__ float bf16_round(float x)
     return __bfloat162float(__float2bfloat16_rn(x));
 }
 
-// One mask nibble (bits b0m..b3m of word w) -> the second-operand registers of a k-step:
+// One mask nibble (bits b0m..b3m of word w) -> the first-operand registers of a k-step for one token:
 //   k0,k1 : the nibble's kept values in dense positions (zero where pruned); `addr` is the shared
 //           address of the token's next unread kept value (rows of 32 bytes) and advances per set bit;
 //   m0,m1 : the nibble as 0/1 in bf16 (1.0 = 0x3F80).
@@ -118,9 +140,10 @@ __device__ __forceinline__ void expand_nibble(unsigned w, unsigned b0m, unsigned
 }
 
 template <int G>
-__global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const DecodeArgs A)
+__global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeArgs A)
 {
     using S = SmemBf16<G>;
+    constexpr bool kShared8 = (G <= 4);        // q' high and low parts share one 8-column operand
     extern __shared__ __align__(128) unsigned char smem[];
     const Ctrl C = make_ctrl(smem);
     unsigned char* tab = smem + S::kTab;
@@ -148,14 +171,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const De
 #else
 #define SPARK_PROBE() do { } while (0)
 #endif
-    if (warp == kConsumerWarps) {
+    if (warp == kNW) {
         producer_loop(A, C, ring, c0, c1, lane);
         return;
     }
-    write_empty_sequences(A, prefix, tid);
+    write_empty_sequences<kNT>(A, prefix, tid);
 
-    const int c = lane & 3, r = lane >> 2;                 // quad lane / fragment row (= token column)
-    const bool row_ok = r < G;
+    const int c = lane & 3, r = lane >> 2;                 // quad lane / fragment row
     int base = 0;
     for (int g = c0; g < c1;) {
         const Segment sg = locate(prefix, A.B, A.Hkv, g, c1);
@@ -191,126 +213,146 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const De
             for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFull, part, o);
             if (lane == 0) qsum_s[warp] = static_cast<float>(part);
         }
-        consumer_sync();
-        // first-operand fragments of this thread: Aq[2s], Aq[2s+1] = q[row r][32c+4s .. +3], same for q' parts
-        unsigned Aq[16], Ahi[16], Alo[16];
-        float qsum = 0.f;
-        if (row_ok) {
-            const unsigned t0 = smem_u32(tab) + r * (kHeadDim * 2) + c * 64;
+        consumer_sync<kNT>();
+        // second-operand fragments (column r of each operand, channels 32c .. 32c+31):
+        //   Bq[2s], Bq[2s+1] = q[head r][32c+4s .. +3];  Bp / Bpl likewise from the q' parts.
+        unsigned Bq[16], Bp[16], Bpl[kShared8 ? 1 : 16];
+        {
+            const unsigned t0 = smem_u32(tab) + c * 64;
+            const unsigned plane = G * kHeadDim * 2;
+            const int pr = kShared8 ? (r & 3) : r;                     // head of column r in the q' operand
+            const unsigned pofs = kShared8 ? ((r < 4) ? plane : 2 * plane) : plane;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 u = lds_u32x4(t0 + i * 16);
-                const uint4 v = lds_u32x4(t0 + G * kHeadDim * 2 + i * 16);
-                const uint4 x = lds_u32x4(t0 + 2 * G * kHeadDim * 2 + i * 16);
-                Aq[4 * i] = u.x; Aq[4 * i + 1] = u.y; Aq[4 * i + 2] = u.z; Aq[4 * i + 3] = u.w;
-                Ahi[4 * i] = v.x; Ahi[4 * i + 1] = v.y; Ahi[4 * i + 2] = v.z; Ahi[4 * i + 3] = v.w;
-                Alo[4 * i] = x.x; Alo[4 * i + 1] = x.y; Alo[4 * i + 2] = x.z; Alo[4 * i + 3] = x.w;
+                uint4 u = make_uint4(0, 0, 0, 0), v = make_uint4(0, 0, 0, 0), x = make_uint4(0, 0, 0, 0);
+                if (r < G) u = lds_u32x4(t0 + r * (kHeadDim * 2) + i * 16);
+                if (pr < G) v = lds_u32x4(t0 + pofs + pr * (kHeadDim * 2) + i * 16);
+                if (!kShared8 && r < G) x = lds_u32x4(t0 + 2 * plane + r * (kHeadDim * 2) + i * 16);
+                Bq[4 * i] = u.x; Bq[4 * i + 1] = u.y; Bq[4 * i + 2] = u.z; Bq[4 * i + 3] = u.w;
+                Bp[4 * i] = v.x; Bp[4 * i + 1] = v.y; Bp[4 * i + 2] = v.z; Bp[4 * i + 3] = v.w;
+                if (!kShared8) { Bpl[4 * i] = x.x; Bpl[4 * i + 1] = x.y; Bpl[4 * i + 2] = x.z; Bpl[4 * i + 3] = x.w; }
             }
-            qsum = qsum_s[r];
-        } else {
+        }
+        // this thread's two heads in the score layout (columns 2c, 2c+1)
+        bool hv[2];
+        float qsum[2];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { Aq[i] = 0; Ahi[i] = 0; Alo[i] = 0; }
+        for (int e = 0; e < 2; ++e) {
+            hv[e] = (2 * c + e < G) && (!kShared8 || c < 2);
+            qsum[e] = hv[e] ? qsum_s[2 * c + e] : 0.f;
         }
         SPARK_PROBE();      // setup done
 
-        float m_run = -INFINITY, l_run = 0.f;
-        float o[16][4];
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float o[8][4];
 #pragma unroll
-        for (int nt = 0; nt < 16; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; o[nt][2] = 0.f; o[nt][3] = 0.f; }
+        for (int mt = 0; mt < 8; ++mt) { o[mt][0] = 0.f; o[mt][1] = 0.f; o[mt][2] = 0.f; o[mt][3] = 0.f; }
 
-        int n = base + ((warp - base) % kConsumerWarps + kConsumerWarps) % kConsumerWarps;
-        for (; n < base + sg.n; n += kConsumerWarps) {
+        int n = base + ((warp - base) % kNW + kNW) % kNW;
+        for (; n < base + sg.n; n += kNW) {
             const int i = sg.i0 + (n - base);
             const int slot = n % NS;
             const bool ok = mbar_wait(&C.full[slot], (n / NS) & 1, C.abort_flag, A.status);
-            const unsigned sbase = ring_u + static_cast<unsigned>(slot) * A.slot_stride;
-            const int n_valid = min(kStepTokens, len - i * kStepTokens);
+            const unsigned page = ring_u + static_cast<unsigned>(slot) * A.slot_stride;
+            const int n_valid = min(kPageTokens, len - i * kPageTokens);
 #ifdef SPARK_CTA_TIMING
             if (tid == 0 && t_first == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_first));
 #endif
             if (ok) {
-#pragma unroll 1
-                for (int pg = 0; pg < 2; ++pg) {
-                    if (pg * kPageTokens >= n_valid) break;                    // warp-uniform
-                    const unsigned page = sbase + pg * L.page_bytes;
-                    // ---------------- scores of the page's 16 tokens ----------------
-                    float accA[2][4], accB[2][4];
-                    unsigned vaddr[2], w[2];
+                // ---------------- scores of the page's 16 tokens (rows r and r+8) ----------------
+                float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f}, d3[4] = {0.f, 0.f, 0.f, 0.f};
+                unsigned vaddr[2], w[2];
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
+                for (int j = 0; j < 2; ++j) {
+                    const int tok = 8 * j + r;
+                    w[j] = lds_u32(page + L.mask_off + tok * 16 + c * 4);
+                    const int cnt = __popc(w[j]);
+                    int x = cnt;
+                    int t = __shfl_up_sync(kFull, x, 1, 4);
+                    if (c >= 1) x += t;
+                    t = __shfl_up_sync(kFull, x, 2, 4);
+                    if (c >= 2) x += t;
+                    vaddr[j] = page + tok * 2 + (x - cnt) * 32;
+                }
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) { accA[j][e] = 0.f; accB[j][e] = 0.f; }
-                        const int tok = 8 * j + r;
-                        w[j] = lds_u32(page + L.mask_off + tok * 16 + c * 4);
-                        const int cnt = __popc(w[j]);
-                        int x = cnt;
-                        int t = __shfl_up_sync(kFull, x, 1, 4);
-                        if (c >= 1) x += t;
-                        t = __shfl_up_sync(kFull, x, 2, 4);
-                        if (c >= 2) x += t;
-                        vaddr[j] = page + tok * 2 + (x - cnt) * 32;
-                    }
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            unsigned k0, k1, m0, m1;
-                            expand_nibble(w[j], 1u << (4 * ks), 2u << (4 * ks), 4u << (4 * ks), 8u << (4 * ks),
-                                          vaddr[j], k0, k1, m0, m1);
-                            mma_bf16(accA[j], Aq[2 * ks], 0u, Aq[2 * ks + 1], 0u, k0, k1);
-                            mma_bf16(accB[j], Ahi[2 * ks], Alo[2 * ks], Ahi[2 * ks + 1], Alo[2 * ks + 1], m0, m1);
-                        }
-                    }
-                    // ---------------- online softmax over the 16 tokens ----------------
-                    float s[2][2];
-                    float mt = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const float2 mu = lds_f32x2(page + L.mu_off + (8 * j + 2 * c) * 4);
-                        const float muv[2] = {mu.x, mu.y};
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int tok = pg * kPageTokens + 8 * j + 2 * c + e;
-                            const float rec = qsum - accB[j][e] - accB[j][2 + e];
-                            const float sv = A.scale_log2e * fmaf(muv[e], rec, accA[j][e]);
-                            s[j][e] = (tok < n_valid) ? sv : -INFINITY;
-                            mt = fmaxf(mt, s[j][e]);
-                        }
-                    }
-                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 1));
-                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 2));
-                    const float m_new = fmaxf(m_run, mt);
-                    const float alpha = exp2f(m_run - m_new);
-                    m_run = m_new;
-                    float hi[2][2], lo[2][2], psum = 0.f;
+                for (int ks = 0; ks < 8; ++ks) {
+                    unsigned k0[2], k1[2], m0[2], m1[2];
 #pragma unroll
                     for (int j = 0; j < 2; ++j)
+                        expand_nibble(w[j], 1u << (4 * ks), 2u << (4 * ks), 4u << (4 * ks), 8u << (4 * ks),
+                                      vaddr[j], k0[j], k1[j], m0[j], m1[j]);
+                    mma_bf16(d1, k0[0], k0[1], k1[0], k1[1], Bq[2 * ks], Bq[2 * ks + 1]);
+                    mma_bf16(d2, m0[0], m0[1], m1[0], m1[1], Bp[2 * ks], Bp[2 * ks + 1]);
+                    if (!kShared8) mma_bf16(d3, m0[0], m0[1], m1[0], m1[1], Bpl[2 * ks], Bpl[2 * ks + 1]);
+                }
+                // kept q' sums of this thread's heads: high part + low part
+                float rk[4];
 #pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const float p = row_ok ? exp2f(s[j][e] - m_new) : 0.f;
-                            psum += p;
-                            hi[j][e] = bf16_round(p);
-                            lo[j][e] = p - hi[j][e];
-                        }
-                    l_run = fmaf(l_run, alpha, psum);
-                    const unsigned P0 = pack_bf16(hi[0][0], hi[0][1]), P1 = pack_bf16(lo[0][0], lo[0][1]);
-                    const unsigned P2 = pack_bf16(hi[1][0], hi[1][1]), P3 = pack_bf16(lo[1][0], lo[1][1]);
-                    if (__any_sync(kFull, alpha != 1.0f)) {
+                for (int e = 0; e < 4; ++e) {
+                    const float other = kShared8 ? __shfl_xor_sync(kFull, d2[e], 2) : d3[e];
+                    rk[e] = d2[e] + other;
+                }
+                // ---------------- online softmax over the 16 tokens ----------------
+                const float mu[2] = {lds_f32(page + L.mu_off + r * 4), lds_f32(page + L.mu_off + (r + 8) * 4)};
+                float s[2][2], alpha[2], ph[2][2], pl[2][2];
 #pragma unroll
-                        for (int nt = 0; nt < 16; ++nt) {
-                            o[nt][0] *= alpha; o[nt][1] *= alpha; o[nt][2] *= alpha; o[nt][3] *= alpha;
+                for (int e = 0; e < 2; ++e) {
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const float sv = A.scale_log2e * fmaf(mu[j], qsum[e] - rk[2 * j + e], d1[2 * j + e]);
+                        s[j][e] = (r + 8 * j < n_valid) ? sv : -INFINITY;
+                    }
+                    float mt = fmaxf(s[0][e], s[1][e]);
+                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 4));
+                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 8));
+                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 16));
+                    const float m_new = fmaxf(m_run[e], mt);
+                    const float al = ex2(m_run[e] - m_new);
+                    alpha[e] = hv[e] ? al : 1.f;
+                    const float p0 = hv[e] ? ex2(s[0][e] - m_new) : 0.f;
+                    const float p1 = hv[e] ? ex2(s[1][e] - m_new) : 0.f;
+                    l_run[e] = fmaf(l_run[e], alpha[e], p0 + p1);
+                    m_run[e] = m_new;
+                    ph[0][e] = bf16_round(p0); pl[0][e] = p0 - ph[0][e];
+                    ph[1][e] = bf16_round(p1); pl[1][e] = p1 - ph[1][e];
+                }
+                // probabilities: score layout (row = token, cols = heads) -> operand layout (k = token, n = col)
+                unsigned pb0, pb1, pc0 = 0, pc1 = 0;
+                {
+                    const unsigned h0 = pack_bf16(ph[0][0], ph[0][1]), h1 = pack_bf16(ph[1][0], ph[1][1]);
+                    const unsigned l0 = pack_bf16(pl[0][0], pl[0][1]), l1 = pack_bf16(pl[1][0], pl[1][1]);
+                    if (kShared8) {                      // columns 4-7 carry the low parts of heads 0-3
+                        const unsigned x0 = __shfl_xor_sync(kFull, l0, 2), x1 = __shfl_xor_sync(kFull, l1, 2);
+                        pb0 = movmatrix_trans(c < 2 ? h0 : x0);
+                        pb1 = movmatrix_trans(c < 2 ? h1 : x1);
+                    } else {
+                        pb0 = movmatrix_trans(h0); pb1 = movmatrix_trans(h1);
+                        pc0 = movmatrix_trans(l0); pc1 = movmatrix_trans(l1);
+                    }
+                }
+                // rescale the running output when a maximum moved (columns 2c, 2c+1 of every tile)
+                {
+                    float a0 = alpha[0], a1 = alpha[1];
+                    if (kShared8) {
+                        const float y0 = __shfl_xor_sync(kFull, a0, 2), y1 = __shfl_xor_sync(kFull, a1, 2);
+                        if (c >= 2) { a0 = y0; a1 = y1; }
+                    }
+                    if (__any_sync(kFull, a0 != 1.0f || a1 != 1.0f)) {
+#pragma unroll
+                        for (int mt = 0; mt < 8; ++mt) {
+                            o[mt][0] *= a0; o[mt][1] *= a1; o[mt][2] *= a0; o[mt][3] *= a1;
                         }
                     }
-                    // ---------------- P.V ----------------
-                    const int mi = lane >> 3, rr = lane & 7;
-                    const unsigned vrow = page + L.v_off + (((mi & 1) << 3) + rr) * (kHeadDim * 2);
+                }
+                // ---------------- P.V: out^T[channel][col] += V^T[channel][token] P^T[token][col] ----------------
+                const int mi = lane >> 3, rr = lane & 7;
+                const unsigned vrow = page + L.v_off + (((mi >> 1) << 3) + rr) * (kHeadDim * 2);
 #pragma unroll
-                    for (int cb = 0; cb < 8; ++cb) {
-                        unsigned vb[4];
-                        ldmatrix_x4_trans(vb, vrow + (((2 * cb + (mi >> 1)) ^ rr) << 4));
-                        mma_bf16(o[2 * cb], P0, P1, P2, P3, vb[0], vb[1]);
-                        mma_bf16(o[2 * cb + 1], P0, P1, P2, P3, vb[2], vb[3]);
-                    }
+                for (int mt = 0; mt < 8; ++mt) {
+                    unsigned a0, a1, a2, a3;
+                    ldmatrix_x4_trans(a0, a1, a2, a3, vrow + (((2 * mt + (mi & 1)) ^ rr) << 4));
+                    mma_bf16(o[mt], a0, a1, a2, a3, pb0, pb1);
+                    if (!kShared8) mma_bf16(o[mt], a0, a1, a2, a3, pc0, pc1);
                 }
             }
             __syncwarp();
@@ -320,21 +362,33 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_bf16_kernel(const De
 
         // ---------------- hand the warp state to the merge ----------------
         {
-            float lsum = l_run;
-            lsum += __shfl_xor_sync(kFull, lsum, 1);
-            lsum += __shfl_xor_sync(kFull, lsum, 2);
-            if (row_ok) {
-                float* mine = merge + (warp * G + r) * kRec;
+            float lsum[2];
 #pragma unroll
-                for (int nt = 0; nt < 16; ++nt)
-                    *reinterpret_cast<float2*>(mine + 8 * nt + 2 * c) =
-                        make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
-                if (c == 0) { mine[kHeadDim] = m_run; mine[kHeadDim + 1] = lsum; }
+            for (int e = 0; e < 2; ++e) {
+                lsum[e] = l_run[e];
+                lsum[e] += __shfl_xor_sync(kFull, lsum[e], 4);
+                lsum[e] += __shfl_xor_sync(kFull, lsum[e], 8);
+                lsum[e] += __shfl_xor_sync(kFull, lsum[e], 16);
             }
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    float v = o[mt][q4];
+                    if (kShared8) v += __shfl_xor_sync(kFull, v, 2);       // high-part column + low-part column
+                    const int e = q4 & 1;
+                    if (hv[e]) merge[(warp * G + 2 * c + e) * kRec + 16 * mt + r + ((q4 >> 1) << 3)] = v;
+                }
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+                if (hv[e] && r == 0) {
+                    merge[(warp * G + 2 * c + e) * kRec + kHeadDim] = m_run[e];
+                    merge[(warp * G + 2 * c + e) * kRec + kHeadDim + 1] = lsum[e];
+                }
         }
-        consumer_sync();
+        consumer_sync<kNT>();
         SPARK_PROBE();      // all warps done
-        merge_and_publish<G>(A, C, merge, sg, tid);
+        merge_and_publish<G, kNW>(A, C, merge, sg, tid);
         SPARK_PROBE();      // published
         g += sg.n;
         base += sg.n;
@@ -358,7 +412,8 @@ static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin,
 {
     DecodeArgs A = A0;
     using S = SmemBf16<G>;
-    A.slot_stride = static_cast<int>(align_up(2 * static_cast<size_t>(A.L.page_bytes), 128));
+    A.pps = 1;
+    A.slot_stride = static_cast<int>(align_up(static_cast<size_t>(A.L.page_bytes), 128));
     int ns = (smem_optin - S::kRing) / A.slot_stride;
     if (ns > kMaxSlots) ns = kMaxSlots;
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
@@ -368,7 +423,7 @@ static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin,
                              static_cast<int>(smem)) != cudaSuccess)
         return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
-    decode_bf16_kernel<G><<<grid, kDecodeThreads, smem, stream>>>(A);
+    decode_bf16_kernel<G><<<grid, kThreads, smem, stream>>>(A);
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
