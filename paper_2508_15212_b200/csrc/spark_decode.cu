@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
         for (; n < base + sg.n; n += kConsumerWarps) {
             const int i = sg.i0 + (n - base);
             const int slot = n % NS;
-            const bool ok = mbar_wait(&C.full[slot], (n / NS) & 1, C.abort_flag, A.status);
+            const bool ok = slot_wait(C.full, C.seq, slot, n / NS, C.abort_flag, A.status);
             const unsigned char* sbase = ring + static_cast<size_t>(slot) * A.slot_stride;
             const int n_valid = min(kStepTokens, len - i * kStepTokens);
             if (ok) {

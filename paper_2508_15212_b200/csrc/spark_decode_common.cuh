@@ -111,6 +111,22 @@ __device__ __forceinline__ uint64_t policy_evict_first()
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
+// Consumer side of a ring slot: wait until the data of revolution `round` has landed in `slot`.
+// A parity wait alone cannot tell "revolution r has not been armed yet" from "revolution r is
+// complete" (consumers of different revolutions of one slot are different warps), so the slot's
+// revolution counter, written by the producer when it arms the barrier, is checked first.
+__device__ __forceinline__ bool slot_wait(uint64_t* full, volatile int* seq, int slot, int round,
+                                          volatile int* abort_flag, int* status)
+{
+    unsigned it = 0;
+    while (seq[slot] != round + 1) {
+        if (++it >= kSpinLimit || *abort_flag) {
+            if (!*abort_flag) { *abort_flag = 1; record_error(status, SPARK_ERR_DEVICE_TIMEOUT); }
+            return false;
+        }
+    }
+    return mbar_wait(&full[slot], round & 1, abort_flag, status);
+}
 template <int NT> __device__ __forceinline__ void consumer_sync()
 {
     asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
@@ -170,6 +186,7 @@ struct Ctrl {
     uint64_t* empty;
     volatile int* abort_flag;
     volatile int* last_flag;
+    volatile int* seq;        // [32] revolution + 1 for which each slot was last armed
     Plan* plan;
     int* prefix;
 };
@@ -182,6 +199,7 @@ __device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
     c.abort_flag = reinterpret_cast<volatile int*>(smem + 512);
     c.last_flag = reinterpret_cast<volatile int*>(smem + 516);
     c.plan = reinterpret_cast<Plan*>(smem + 528);
+    c.seq = reinterpret_cast<volatile int*>(smem + 640);
     c.prefix = reinterpret_cast<int*>(smem + kCtrlBytes);
     return c;
 }
@@ -192,6 +210,7 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
 {
     const int warp = tid >> 5, lane = tid & 31;
     const int max_tokens = A.max_blocks * kPageTokens;
+    if (warp == 1) C.seq[lane] = 0;
     if (tid == 32) {
         for (int s = 0; s < A.nslots; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], 1); }
         *C.abort_flag = 0;
@@ -325,6 +344,7 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
         while (__any_sync(kFull, pending)) {
             if (pending && (round == 0 || mbar_try_wait(empty, (round - 1) & 1))) {
                 const unsigned bytes = L.page_bytes * (cur1 >= 0 ? 2u : 1u);
+                C.seq[lane] = round + 1;
                 mbar_expect_tx(full, bytes);
                 bulk_g2s(dst, A.pages + static_cast<int64_t>(cur0) * L.page_bytes, L.page_bytes, full, policy);
                 if (cur1 >= 0)

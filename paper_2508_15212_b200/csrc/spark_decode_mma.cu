@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
         for (; n < base + sg.n; n += kNW) {
             const int i = sg.i0 + (n - base);
             const int slot = n % NS;
-            const bool ok = mbar_wait(&C.full[slot], (n / NS) & 1, C.abort_flag, A.status);
+            const bool ok = slot_wait(C.full, C.seq, slot, n / NS, C.abort_flag, A.status);
             const unsigned page = ring_u + static_cast<unsigned>(slot) * A.slot_stride;
             const int n_valid = min(kPageTokens, len - i * kPageTokens);
 #ifdef SPARK_CTA_TIMING
