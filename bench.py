@@ -345,7 +345,7 @@ def main():
             "gpu_launches": args.steps * B.spark_last_launch_count(),
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(name),
-                         "kernel": "spark::decode_kernel", "algorithmic_bytes_per_launch": alg_bytes},
+                         "kernel": "spark::decode_bf16_kernel" if wl.dtype == "bf16" else "spark::decode_f32_kernel", "algorithmic_bytes_per_launch": alg_bytes},
             "cpu_baseline": cpu_baseline,
             "compress": {"us": compress_us, "gbs": compress_bytes / (compress_us * 1e-6) / 1e9,
                          "bytes": compress_bytes, "launches": 2},
