@@ -154,6 +154,32 @@ spark_status spark_decode_attn(const spark_params *p, const void *q,
                                void *workspace, size_t workspace_bytes, spark_stream_t stream);
 
 /*
+ * spark_decode_attn_noalloc -- spark_decode_attn for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the call above, same arithmetic.)
+ *
+ * Who needs it: code that is handed device tensors but no allocator -- a serving loop whose memory
+ * was divided up once at start-up, a plug-in inside another runtime, a framework section in which
+ * cudaMalloc is forbidden.  Such a caller can supply inputs and outputs but not the scratch that split
+ * decoding needs, so this variant uses a fixed scratch array that lives in the library's own device
+ * image (about 1.3 MB per GPU that loads the library, held until the process exits).  It calls no
+ * cudaMalloc, cudaFree or allocating library routine.
+ *
+ *   - Limit: batch * n_kv_heads <= 64 (any group size up to 8).  Larger problems are refused with
+ *     SPARK_ERR_WORKSPACE before anything is enqueued; use spark_decode_attn with your own workspace.
+ *   - The first call on each device looks up the array's device address (the device must be current).
+ *     Make that first call outside any stream capture.
+ *   - Every call shares the one array.  The entry point clears the status word and the tickets on the
+ *     stream before launching; two calls that overlap on the GPU (different streams, no dependency)
+ *     would race on it and are not supported.  Device-side errors are not readable through
+ *     spark_read_status for this variant (there is no caller-visible workspace).
+ *   - All other arguments, results and error codes are those of spark_decode_attn.
+ */
+spark_status spark_decode_attn_noalloc(const spark_params *p, const void *q,
+                                       const void *pages, const int32_t *block_table, int32_t max_blocks,
+                                       const int32_t *packed_lens, const float *qnorm,
+                                       float *out, float *lse, spark_stream_t stream);
+
+/*
  * spark_unpack_pages -- pages back to logical arrays (what the paper calls the pruned
  * key matrix K^, the mask S and mu_pruned; Sec. "Saliency Measurement and Unstructured
  * Pruning").  For inspection and tests; any output may be NULL.

@@ -22,7 +22,8 @@ SPARK_F32, SPARK_BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
-           "spark_compress", "spark_decode_attn", "spark_unpack_pages", "spark_read_status"]
+           "spark_compress", "spark_decode_attn", "spark_decode_attn_noalloc", "spark_unpack_pages",
+           "spark_read_status"]
 
 
 class SparkError(RuntimeError):
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.spark_compress.argtypes = [P, vp, vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.spark_decode_attn.restype = i32
         L.spark_decode_attn.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spark_decode_attn_noalloc.restype = i32
+        L.spark_decode_attn_noalloc.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.spark_unpack_pages.restype = i32
         L.spark_unpack_pages.argtypes = [P, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp]
         L.spark_read_status.restype = i32
@@ -145,6 +148,14 @@ def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm
                                    block_table.shape[-1], _ptr(packed_lens), _ptr(qnorm), _ptr(out), _ptr(lse),
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
            "spark_decode_attn")
+
+
+def spark_decode_attn_noalloc(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse) -> None:
+    """Decode step that brings its own fixed scratch (batch * n_kv_heads <= 64); allocates nothing."""
+    _check(lib().spark_decode_attn_noalloc(ctypes.byref(p), _ptr(q), _ptr(pages), _ptr(block_table),
+                                           block_table.shape[-1], _ptr(packed_lens), _ptr(qnorm), _ptr(out),
+                                           _ptr(lse), _stream()),
+           "spark_decode_attn_noalloc")
 
 
 def spark_unpack_pages(p: spark_params, pages, block_table, packed_lens, max_tokens, mask=None, mu=None,

@@ -7,7 +7,7 @@ using namespace spark;
 
 static thread_local int g_last_launches = 0;
 
-static spark_status check_params(const spark_params* p)
+spark_status spark::check_params(const spark_params* p)
 {
     if (!p) return SPARK_ERR_NULL;
     if (p->head_dim != kHeadDim || p->page_tokens != kPageTokens) return SPARK_ERR_UNSUPPORTED;

@@ -84,6 +84,9 @@ template <> struct Elem<__nv_bfloat16> {
     }
 };
 
+// host-side validation of a parameter block (spark_api.cu)
+spark_status check_params(const spark_params* p);
+
 // ---- host-side launchers implemented in the .cu files -------------------------------------------
 spark_status launch_compress(const spark_params& p, const void* q_win, const void* k, const void* v,
                              int64_t sb, int64_t sh, int64_t st, const int32_t* seq_lens,

@@ -1,0 +1,60 @@
+"""The allocation-free decode entry point against the regular one.
+
+spark_decode_attn_noalloc serves callers that are handed device tensors but may not allocate (no
+workspace to pass): it runs the same kernels on a scratch array built into the library.  The check: on
+the same packed cache its output equals the regular entry point's (same tolerance as the parity tests),
+on two calls in a row (the second call finds the scratch as the first left it), and problems beyond the
+built-in scratch are refused before anything is launched.  Collected last on purpose.
+"""
+import pytest
+import torch
+
+from paper_2508_15212_b200 import binding as B
+from paper_2508_15212_b200 import build as spark_build
+from paper_2508_15212_b200 import inputs
+from paper_2508_15212_b200.cache import SparkCache
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-5, "bf16": 2e-3}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    spark_build.build()
+    B.lib()
+
+
+@pytest.mark.parametrize("dtype,Bn,Hq,Hkv,lens,keep", [
+    ("bf16", 2, 16, 4, [2100, 333], 64),        # several CTAs share a unit: partials and tickets in use
+    ("bf16", 1, 28, 4, [5000], 38),
+    ("f32", 2, 4, 2, [700, 64], 25),
+])
+def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, keep):
+    wl = inputs.make_workload(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=lens, window=16, dtype=dtype,
+                              sigma_s=1.0 if dtype == "bf16" else 0.5, seed=321, device="cuda")
+    cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=16, keep=keep, dtype=dtype,
+                       max_tokens=max(lens))
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    lse_ref = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
+    ref = cache.decode(wl.q, lse=lse_ref)
+    assert cache.status() == 0
+    for call in range(2):
+        out = torch.full((Bn, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
+        lse = torch.full((Bn, Hq), float("nan"), dtype=torch.float32, device="cuda")
+        B.spark_decode_attn_noalloc(cache.params, wl.q, cache.pages, cache.block_table, cache.packed_lens,
+                                    cache.qnorm, out, lse)
+        torch.cuda.synchronize()
+        d = float((out - ref).abs().max())
+        assert d <= TOL[dtype], f"call {call}: max|delta| {d:.3e}"
+        assert float((lse - lse_ref).abs().max()) <= 1e-3
+
+
+def test_noalloc_refuses_problems_beyond_its_scratch():
+    p = B.make_params(batch=65, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype=torch.bfloat16,
+                      n_pool_pages=65)
+    dummy = torch.zeros(1 << 12, dtype=torch.uint8, device="cuda")
+    bt = torch.zeros(65, 1, 1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.SparkError) as e:
+        B.spark_decode_attn_noalloc(p, dummy, dummy, bt, dummy, dummy, dummy, None)
+    assert e.value.code == 4            # SPARK_ERR_WORKSPACE, nothing launched
