@@ -104,6 +104,10 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
                            size_t workspace_bytes, cudaStream_t stream, int* launches);
 
 size_t decode_workspace_bytes(const spark_params& p);
+size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens);
+spark_status launch_evict(const spark_params& p, const void* q_win, const void* k, int64_t sb, int64_t sh,
+                          int64_t st, const int32_t* seq_lens, int32_t max_seq_tokens, int32_t* packed_lens,
+                          int32_t* kept_tokens, void* workspace, cudaStream_t stream, int* launches);
 size_t compress_workspace_bytes(const spark_params& p, int64_t max_seq_tokens);
 
 }  // namespace spark

@@ -271,10 +271,7 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
 // ------------------------------------------------------------------------------------------------
 size_t compress_workspace_bytes(const spark_params& p, int64_t max_seq_tokens)
 {
-    size_t bytes = kWorkspaceHeader;
-    (void)max_seq_tokens;
-    (void)p;
-    return bytes;
+    return kWorkspaceHeader + evict_workspace_bytes(p, max_seq_tokens);
 }
 
 spark_status launch_compress(const spark_params& p, const void* q_win, const void* k, const void* v,
@@ -284,25 +281,30 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
                              void* workspace, size_t workspace_bytes, cudaStream_t stream, int* launches)
 {
     (void)workspace_bytes;
-    (void)kept_tokens;
-    if (p.token_budget > 0) return SPARK_ERR_UNSUPPORTED;
     int* status = static_cast<int*>(workspace);
+    const bool evict = p.token_budget > 0;
+    if (evict) {            // writes kept_tokens and packed_lens
+        const spark_status st_e = launch_evict(p, q_win, k, sb, sh, st, seq_lens, max_seq_tokens, packed_lens,
+                                               kept_tokens, workspace, stream, launches);
+        if (st_e != SPARK_OK) return st_e;
+    }
     const float eps = p.qnorm_eps > 0.f ? p.qnorm_eps : 1e-12f;
     const dim3 qgrid(p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16)
         window_qnorm_kernel<__nv_bfloat16><<<qgrid, kHeadDim, 0, stream>>>(
-            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, packed_lens, max_seq_tokens, status);
+            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, evict ? nullptr : packed_lens, max_seq_tokens, status);
     else
         window_qnorm_kernel<float><<<qgrid, kHeadDim, 0, stream>>>(
-            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, packed_lens, max_seq_tokens, status);
+            q_win, p.n_q_heads, p.n_kv_heads, p.window, eps, qnorm, seq_lens, evict ? nullptr : packed_lens, max_seq_tokens, status);
     ++*launches;
     if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
 
-    const int n_blocks = (max_seq_tokens + kPageTokens - 1) / kPageTokens;
+    const int max_packed = (evict && p.token_budget < max_seq_tokens) ? p.token_budget : max_seq_tokens;
+    const int n_blocks = (max_packed + kPageTokens - 1) / kPageTokens;
     if (n_blocks == 0) return SPARK_OK;
     CompressArgs A;
     A.k = k; A.v = v; A.sb = sb; A.sh = sh; A.st = st;
-    A.lens = packed_lens; A.gather = nullptr; A.gather_stride = 0;
+    A.lens = packed_lens; A.gather = evict ? kept_tokens : nullptr; A.gather_stride = evict ? p.token_budget : 0;
     A.qnorm = qnorm; A.pages = static_cast<unsigned char*>(pages);
     A.block_table = block_table; A.max_blocks = max_blocks; A.Hkv = p.n_kv_heads; A.keep = p.keep;
     A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep); A.status = status;

@@ -162,3 +162,62 @@ def test_bad_page_id_is_recorded_not_dereferenced():
     cache.block_table[0, 0, 1] = 1 << 20                       # outside the pool
     cache.decode(wl.q)
     assert B.spark_read_status(cache.ws_decode) == 6            # SPARK_ERR_DEVICE_BOUNDS
+
+
+def evicted_reference(wl_cpu, budget, pool, keep):
+    """Oracle side of eviction + pruning + decode: returns kept tokens, lengths, boundary gaps, output."""
+    Bn, Hq, Hkv, W, D, S = wl_cpu.shape
+    lens = wl_cpu.seq_lens.tolist()
+    kept, n, vote, pooled = oracle.evict(wl_cpu.q_win, wl_cpu.k, lens, budget, pool, want_votes=True)
+    gaps = np.full((Bn, Hkv), np.inf)
+    for b in range(Bn):
+        if lens[b] <= budget:
+            continue
+        P, k = lens[b] - W, budget - W
+        for h in range(Hkv):
+            srt = np.sort(pooled[b, h, :P])[::-1]
+            gaps[b, h] = (srt[k - 1] - srt[k]) / max(srt[k - 1], 1e-300)
+    kk, vv = to_np(wl_cpu.k), to_np(wl_cpu.v)
+    kg, vg = np.zeros((Bn, Hkv, budget, D), kk.dtype), np.zeros((Bn, Hkv, budget, D), vv.dtype)
+    for b in range(Bn):
+        for h in range(Hkv):
+            idx = kept[b, h, :n[b]]
+            kg[b, h, :n[b]] = kk[b, h, idx]
+            vg[b, h, :n[b]] = vv[b, h, idx]
+    _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
+    c = oracle.compress(kg, n, keep, a)
+    out, _ = oracle.decode_attn(to_np(wl_cpu.q), kg, vg, n, c["mask"], c["mu"], a)
+    return kept, n, gaps, c, out
+
+
+@pytest.mark.parametrize("dtype,lens,W,budget,G", [("bf16", [600, 90, 300], 8, 128, 4),
+                                                   ("bf16", [2000], 32, 256, 7),
+                                                   ("f32", [500, 64], 16, 96, 2)])
+def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
+    keep, Hkv, Bn = 64, 2, len(lens)
+    wl = make(dtype, Bn, Hkv * G, Hkv, lens, W, keep, seed=130 + G, sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
+    wl_cpu = wl.to("cpu")
+    kept_ref, n_ref, gaps, c_ref, out_ref = evicted_reference(wl_cpu, budget, 7, keep)
+    cache = SparkCache(batch=Bn, n_q_heads=Hkv * G, n_kv_heads=Hkv, window=W, keep=keep, dtype=dtype,
+                       max_tokens=max(lens), token_budget=budget, pool_kernel=7)
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    assert cache.status() == 0
+    assert cache.packed_lens.cpu().tolist() == n_ref.tolist()
+    kept = cache.kept_tokens.cpu().numpy()
+    same = True
+    for b in range(Bn):
+        for h in range(Hkv):
+            a_, r_ = kept[b, h, :n_ref[b]], kept_ref[b, h, :n_ref[b]]
+            assert (np.diff(a_) > 0).all() and a_[-W:].tolist() == list(range(lens[b] - W, lens[b]))
+            if gaps[b, h] > 1e-4:
+                assert np.array_equal(a_, r_), f"evicted set differs at unit ({b},{h}), gap {gaps[b, h]:.2e}"
+            else:
+                same = same and np.array_equal(a_, r_)
+                assert len(set(a_.tolist()) & set(r_.tolist())) >= n_ref[b] - 2
+    if same:
+        u = cache.unpack(want_vals=False, want_v=False)
+        assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c_ref["mask"])
+        out = cache.decode(wl.q)
+        assert cache.status() == 0
+        d = float(np.abs(out.cpu().numpy() - out_ref).max())
+        assert d <= TOL[dtype], f"max|delta| {d:.3e}"
