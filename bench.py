@@ -163,6 +163,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="index into the benchmark configurations (0-based)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--keep", type=int, default=0, help="override the kept-channel count T")
+    ap.add_argument("--ratio", type=float, default=None, help="pruning ratio (configuration 5 sweeps 0.3/0.5/0.7/0.8)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
 
@@ -170,6 +171,8 @@ def main():
     from paper_2508_15212_b200 import inputs
     cfg = dict(inputs.CONFIGS[args.config])
     ratio = cfg["ratio"] if not isinstance(cfg["ratio"], tuple) else cfg["ratio"][1]
+    if args.ratio is not None:
+        ratio = args.ratio
     cfg["ratio"] = ratio
     keep = args.keep or inputs.keep_count(cfg["head_dim"], ratio)
     if isinstance(cfg["seq_lens"], tuple):
@@ -183,16 +186,12 @@ def main():
     from paper_2508_15212_b200 import build as spark_build
     from paper_2508_15212_b200.cache import SparkCache
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2508_15212_b200 import dist_utils
+    rank, world, local = dist_utils.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist = dist_utils.init_process_group("nccl", torch.device("cuda", local))
     if rank == 0:
         spark_build.build()
     if dist is not None:
@@ -200,37 +199,75 @@ def main():
     B.lib()
 
     # ---- workload (weak scaling: every rank holds its own copy of the configuration) ----
-    wl = inputs.config_workload(args.config, device="cuda", seed_offset=rank)
-    inputs.enforce_saliency_gap(wl, keep)
-    Bn, Hq, Hkv, W, D, S = wl.shape
-    lens = wl.seq_lens.tolist()
+    # A step is a list of (cache, q, out) decode launches: one for the single-layer configurations
+    # (rotating over cold copies), 28 (one per layer) for the Qwen-shaped configuration.
+    from paper_2508_15212_b200.cache import build_evicted_batch, permuted_block_table
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
-    mk = lambda: SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
-                            max_tokens=S)
-    first = mk()
-    alg_bytes = first.algorithmic_bytes_per_token * Hkv * sum(lens)
-    copies = max(1, min(64, -(-4 * l2 // max(alg_bytes, 1))))
-    caches = [first] + [mk() for _ in range(copies - 1)]
-
-    # compress (prefill side): timed for information
+    D = cfg["head_dim"]
+    esize = 2 if cfg["dtype"] == "bf16" else 4
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    for c in caches:
-        c.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
-    torch.cuda.synchronize()
-    ev[0].record()
-    for c in caches:
-        c.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
-    ev[1].record()
-    torch.cuda.synchronize()
-    compress_us = ev[0].elapsed_time(ev[1]) * 1e3 / len(caches)
-    e = 2 if wl.dtype == "bf16" else 4
-    compress_bytes = Hkv * sum(lens) * (2 * D * e + first.page_bytes // 16)
-
-    out = torch.empty(Bn, Hq, D, dtype=torch.float32, device="cuda")
+    wl = None
+    step_sets = []                     # step i uses step_sets[i % len(step_sets)]
+    compress_us = compress_bytes = None
+    if "token_budget" in cfg:          # prompts evicted and pruned one at a time into one batch cache
+        per_tok = B.spark_algorithmic_bytes_per_token(B.make_params(
+            batch=1, n_q_heads=cfg["n_q_heads"], n_kv_heads=cfg["n_kv_heads"], window=cfg["window"], keep=keep,
+            dtype=torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32, n_pool_pages=1))
+        alg_bytes = per_tok * cfg["n_kv_heads"] * cfg["token_budget"] * cfg["batch"]
+        copies = max(1, -(-4 * l2 // alg_bytes))
+        for c in range(copies):
+            cache, q, _, _ = build_evicted_batch(cfg, keep, seed_offset=dist_utils.rank_seed_offset(rank, c))
+            out = torch.empty(cfg["batch"], cfg["n_q_heads"], D, dtype=torch.float32, device="cuda")
+            step_sets.append([(cache, q, out)])
+        cfg["cached_tokens_after_eviction"] = cfg["token_budget"]
+    elif "n_layers" in cfg:            # paged pool, variable lengths, all layers per step
+        copies, alg_bytes, layer_set = 1, 0, []
+        for layer in range(cfg["n_layers"]):
+            wl_l = inputs.config_workload(args.config, device="cuda", seed_offset=dist_utils.rank_seed_offset(rank, layer))
+            Bn, Hq, Hkv, W, _, S = wl_l.shape
+            lens = wl_l.seq_lens.tolist()
+            table, n_pages = permuted_block_table(Bn, Hkv, lens, "cuda", seed=977 * layer + rank)
+            cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl_l.dtype,
+                               max_tokens=S, block_table=table, n_pool_pages=n_pages)
+            cache.compress(wl_l.q_win, wl_l.k, wl_l.v, wl_l.seq_lens)
+            alg_bytes += cache.algorithmic_bytes_per_token * Hkv * sum(lens)
+            layer_set.append((cache, wl_l.q.clone(), torch.empty(Bn, Hq, D, dtype=torch.float32, device="cuda")))
+            total_tokens = locals().get("total_tokens", 0) + sum(lens)
+            del wl_l
+            torch.cuda.empty_cache()
+        step_sets.append(layer_set)
+        cfg["seq_lens"] = (f"uniform[8192,131072] per sequence, independent per layer; "
+                           f"{total_tokens} tokens over {cfg['n_layers']} layers")
+    else:
+        wl = inputs.config_workload(args.config, device="cuda", seed_offset=dist_utils.rank_seed_offset(rank))
+        inputs.enforce_saliency_gap(wl, keep)
+        Bn, Hq, Hkv, W, _, S = wl.shape
+        lens = wl.seq_lens.tolist()
+        mk = lambda: SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
+                                max_tokens=S)
+        first = mk()
+        alg_bytes = first.algorithmic_bytes_per_token * Hkv * sum(lens)
+        copies = max(1, min(64, -(-4 * l2 // max(alg_bytes, 1))))
+        caches = [first] + [mk() for _ in range(copies - 1)]
+        for c in caches:               # compress (prefill side): timed for information
+            c.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+        torch.cuda.synchronize()
+        ev[0].record()
+        for c in caches:
+            c.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+        ev[1].record()
+        torch.cuda.synchronize()
+        compress_us = ev[0].elapsed_time(ev[1]) * 1e3 / len(caches)
+        compress_bytes = Hkv * sum(lens) * (2 * D * esize + first.page_bytes // 16)
+        out = torch.empty(Bn, Hq, D, dtype=torch.float32, device="cuda")
+        step_sets = [[(c, wl.q, out)] for c in caches]
+    launches_per_step = len(step_sets[0])
+    first = step_sets[0][0][0]
     stream = torch.cuda.Stream()
 
     def launch(i):
-        caches[i % copies].decode(wl.q, out=out)
+        for cache, q, out in step_sets[i % len(step_sets)]:
+            cache.decode(q, out=out)
 
     # ---- graphs of decode launches ----
     def capture(n):
@@ -244,7 +281,7 @@ def main():
         for i in range(max(args.warmup, 3)):
             launch(i)
     stream.synchronize()
-    spg = min(args.steps, 20 * copies)
+    spg = min(args.steps, max(1, (20 * len(step_sets)) // launches_per_step))
     g_main = capture(spg)
     n_rep, rem = divmod(args.steps, spg)
     g_rem = capture(rem) if rem else None
@@ -281,29 +318,29 @@ def main():
                 with torch.cuda.stream(stream):
                     g_main.replay()
                 stream.synchronize()
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = dist_utils.max_over_ranks(ms, dist, "cuda")
     us_step = ms * 1e3 / args.steps
     status = first.status()
 
     # ---- end to end through the public call: pinned host q -> device, decode, out -> pinned host ----
-    q_host = wl.q.cpu().pin_memory()
-    out_host = torch.empty(Bn, Hq, D, dtype=torch.float32).pin_memory()
-    q_dev = torch.empty_like(wl.q)
-    e2e_steps = min(args.steps, 500)
+    host = [[(q.cpu().pin_memory(), torch.empty(out.shape, dtype=torch.float32).pin_memory(), torch.empty_like(q))
+             for _, q, out in st] for st in step_sets]
+    h2d = sum(qh.numel() * qh.element_size() for qh, _, _ in host[0])
+    d2h = sum(oh.numel() * 4 for _, oh, _ in host[0])
+    e2e_steps = min(args.steps, 500 if launches_per_step == 1 else 50)
+
     def e2e_step(i):
-        q_dev.copy_(q_host, non_blocking=True)
-        caches[i % copies].decode(q_dev, out=out)
-        out_host.copy_(out, non_blocking=True)
+        k = i % len(step_sets)
+        for (cache, _, out), (qh, oh, qd) in zip(step_sets[k], host[k]):
+            qd.copy_(qh, non_blocking=True)
+            cache.decode(qd, out=out)
+            oh.copy_(out, non_blocking=True)
         torch.cuda.current_stream().synchronize()
     for i in range(5):
         e2e_step(i)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    t0 = time.perf_counter()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(e2e_steps):
@@ -311,20 +348,17 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = dist_utils.max_over_ranks(e2e_ms, dist, "cuda")
     e2e_us = e2e_ms * 1e3 / e2e_steps
 
     # ---- oracle on the host cores (rank 0, N = 1 only) ----
     cpu_baseline, max_err = None, None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and wl is not None:
         wl_cpu = wl.to("cpu")
         t_or, cores, o_ref = oracle_decode_time(wl_cpu, keep)
         cpu_baseline = {"value": t_or * 1e6, "unit": "us/step", "cores": cores, "kind": "oracle",
                         "sample": "one full decode step of the workload, median of 3"}
-        max_err = float((caches[0].decode(wl.q).cpu().numpy() - o_ref).__abs__().max())
+        max_err = float((first.decode(wl.q).cpu().numpy() - o_ref).__abs__().max())
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -333,22 +367,26 @@ def main():
         line = {
             "metric": METRIC, "value": us_step, "unit": "us/step", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": us_step / 1e3, "higher_is_better": False,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": wl.dtype, "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": cfg["dtype"], "data": "synthetic",
             "config": workload_desc(cfg, keep, copies),
-            "hbm_gbs": gbs, "hbm_gbs_all_gpus": gbs * world,
+            "hbm_gbs": gbs, "hbm_gbs_all_gpus": dist_utils.aggregate_throughput(alg_bytes / 1e9, world, us_step * 1e-6),
             "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
             "algorithmic_bytes_per_step": alg_bytes,
             "clocks": sampler.summary(),
-            "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": q_host.numel() * q_host.element_size(),
-                    "d2h_bytes_per_step": out_host.numel() * 4, "steps": e2e_steps,
+            "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "note": "packed cache resident; per step: pinned q -> device, spark_decode_attn, out -> pinned host, sync"},
-            "gpu_launches": args.steps * B.spark_last_launch_count(),
+            "gpu_launches": args.steps * launches_per_step * B.spark_last_launch_count(),
+            "launches_per_step": launches_per_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(name),
-                         "kernel": "spark::decode_bf16_kernel" if wl.dtype == "bf16" else "spark::decode_f32_kernel", "algorithmic_bytes_per_launch": alg_bytes},
+                         "kernel": "spark::decode_bf16_kernel" if cfg["dtype"] == "bf16" else "spark::decode_f32_kernel",
+                         "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
+                         "avg_launch_us": us_step / launches_per_step},
             "cpu_baseline": cpu_baseline,
-            "compress": {"us": compress_us, "gbs": compress_bytes / (compress_us * 1e-6) / 1e9,
-                         "bytes": compress_bytes, "launches": 2},
+            "compress": None if compress_us is None else {
+                "us": compress_us, "gbs": compress_bytes / (compress_us * 1e-6) / 1e9, "bytes": compress_bytes,
+                "launches": 2},
             "max_abs_err_vs_oracle": max_err, "device_status": status,
         }
         print(json.dumps(line))
