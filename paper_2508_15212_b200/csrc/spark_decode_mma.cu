@@ -249,10 +249,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
         for (int mt = 0; mt < 8; ++mt) { o[mt][0] = 0.f; o[mt][1] = 0.f; o[mt][2] = 0.f; o[mt][3] = 0.f; }
 
         int n = base + ((warp - base) % kNW + kNW) % kNW;
-        for (; n < base + sg.n; n += kNW) {
+        int slot = n % NS, round = n / NS;                 // ring position of step n, kept incrementally
+        for (; n < base + sg.n; n += kNW, slot += kNW) {
+            while (slot >= NS) { slot -= NS; ++round; }
             const int i = sg.i0 + (n - base);
-            const int slot = n % NS;
-            const bool ok = slot_wait(C.full, C.seq, slot, n / NS, C.abort_flag, A.status);
+            const bool ok = slot_wait(C.full, C.seq, slot, round, C.abort_flag, A.status);
             const unsigned page = ring_u + static_cast<unsigned>(slot) * A.slot_stride;
             const int n_valid = min(kPageTokens, len - i * kPageTokens);
 #ifdef SPARK_CTA_TIMING
