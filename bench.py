@@ -165,6 +165,7 @@ def main():
     ap.add_argument("--keep", type=int, default=0, help="override the kept-channel count T")
     ap.add_argument("--ratio", type=float, default=None, help="pruning ratio (configuration 5 sweeps 0.3/0.5/0.7/0.8)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     args = ap.parse_args()
 
     import torch
@@ -173,6 +174,8 @@ def main():
     ratio = cfg["ratio"] if not isinstance(cfg["ratio"], tuple) else cfg["ratio"][1]
     if args.ratio is not None:
         ratio = args.ratio
+    if args.batch:
+        cfg["batch"] = args.batch
     cfg["ratio"] = ratio
     keep = args.keep or inputs.keep_count(cfg["head_dim"], ratio)
     if isinstance(cfg["seq_lens"], tuple):
@@ -239,7 +242,8 @@ def main():
         cfg["seq_lens"] = (f"uniform[8192,131072] per sequence, independent per layer; "
                            f"{total_tokens} tokens over {cfg['n_layers']} layers")
     else:
-        wl = inputs.config_workload(args.config, device="cuda", seed_offset=dist_utils.rank_seed_offset(rank))
+        wl = inputs.config_workload(args.config, device="cuda", seed_offset=dist_utils.rank_seed_offset(rank),
+                                    batch=cfg["batch"])
         inputs.enforce_saliency_gap(wl, keep)
         Bn, Hq, Hkv, W, _, S = wl.shape
         lens = wl.seq_lens.tolist()

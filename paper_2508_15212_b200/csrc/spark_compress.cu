@@ -28,7 +28,15 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
     double acc = 0.0;
     for (int g = 0; g < G; ++g) {
         const int64_t base = ((static_cast<int64_t>(b) * Hq + (h * G + g)) * W) * kHeadDim + j;
-        for (int w = 0; w < W; ++w)
+        int w = 0;
+        for (; w + 8 <= W; w += 8) {                       // eight loads in flight, summed in order
+            float x[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) x[u] = Elem<E>::load(q_win, base + static_cast<int64_t>(w + u) * kHeadDim);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc += static_cast<double>(x[u]);
+        }
+        for (; w < W; ++w)
             acc += static_cast<double>(Elem<E>::load(q_win, base + static_cast<int64_t>(w) * kHeadDim));
     }
     const float m = static_cast<float>(acc / static_cast<double>(G * W));
@@ -121,32 +129,45 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
             key[i] = __float_as_uint(w[i]);
         }
-        // T-th largest key by radix descent
-        unsigned thr = 0;
-        for (int bit = 30; bit >= 0; --bit) {
+        // T-th largest key by radix descent over the bits in which the 128 keys differ.  The descent
+        // stops as soon as a candidate threshold has exactly T keys at or above it (then those are the
+        // kept set and no tie can straddle the boundary); otherwise it ends with the exact T-th largest
+        // key and equal keys are admitted in ascending channel order.
+        const unsigned k_or = __reduce_or_sync(kFullMask, key[0] | key[1] | key[2] | key[3]);
+        const unsigned k_and = __reduce_and_sync(kFullMask, key[0] & key[1] & key[2] & key[3]);
+        const unsigned diff = k_or ^ k_and;
+        const int top = diff ? (31 - __clz(diff)) : -1;              // highest bit in which keys differ
+        unsigned thr = (top >= 0) ? (k_and & ~((2u << top) - 1u)) : k_and;   // common leading bits
+        bool exact = false;
+        for (int bit = top; bit >= 0; --bit) {
             const unsigned cand = thr | (1u << bit);
-            int cnt = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) cnt += __popc(__ballot_sync(kFullMask, key[i] >= cand));
+            const int mine = (key[0] >= cand) + (key[1] >= cand) + (key[2] >= cand) + (key[3] >= cand);
+            const int cnt = __reduce_add_sync(kFullMask, mine);
             if (cnt >= T) thr = cand;
+            if (cnt == T) { exact = true; break; }
         }
-        unsigned eqb[4];
-        int c_gt = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            c_gt += __popc(__ballot_sync(kFullMask, key[i] > thr));
-            eqb[i] = __ballot_sync(kFullMask, key[i] == thr);
-        }
-        const int need_eq = T - c_gt;
-        int rank = 0;                                            // equal keys on lower channels
-#pragma unroll
-        for (int i = 0; i < 4; ++i) rank += __popc(eqb[i] & lt);
         bool kept[4];
+        if (exact) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const bool eq = key[i] == thr;
-            kept[i] = key[i] > thr || (eq && rank < need_eq);
-            rank += eq ? 1 : 0;
+            for (int i = 0; i < 4; ++i) kept[i] = key[i] >= thr;
+        } else {
+            unsigned eqb[4];
+            int c_gt = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                c_gt += __popc(__ballot_sync(kFullMask, key[i] > thr));
+                eqb[i] = __ballot_sync(kFullMask, key[i] == thr);
+            }
+            const int need_eq = T - c_gt;
+            int rank = 0;                                        // equal keys on lower channels
+#pragma unroll
+            for (int i = 0; i < 4; ++i) rank += __popc(eqb[i] & lt);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool eq = key[i] == thr;
+                kept[i] = key[i] > thr || (eq && rank < need_eq);
+                rank += eq ? 1 : 0;
+            }
         }
         // slot of each kept channel = kept channels below it
         int slot = 0;
