@@ -68,7 +68,20 @@ typedef struct {
     float   qnorm_eps;      /* floor of |mean window query|; 0 selects 1e-12                  */
     float   softmax_scale;  /* 0 selects 1/sqrt(head_dim)                                     */
     int64_t n_pool_pages;   /* pages in the pool; every block-table entry must be below it    */
+    int32_t flags;          /* bit set of spark_flags (0: none)                               */
+    int32_t reserved;       /* must be 0                                                      */
 } spark_params;
+
+/* spark_params.flags */
+typedef enum {
+    /* spark_decode_attn only.  Launch the step so that it may begin while the kernel enqueued before it
+     * on the same stream is still draining (programmatic dependent launch): the page stream -- pages,
+     * block table, packed_lens -- is read at once, while q, qnorm, out, lse and the workspace are touched
+     * only after that preceding kernel has completed.  Set it only when the preceding kernel does not
+     * write the packed cache, the block table or packed_lens (a projection that produces q is fine).
+     * Results are identical with and without the flag. */
+    SPARK_FLAG_OVERLAP_PREVIOUS = 1
+} spark_flags;
 
 /* T = floor((1 - ratio) * head_dim): the paper's kept-channel count (Sec. "Problem
  * Formulation", below Eq. (cal)).  Host only.  Returns -1 for ratio outside [0, 1). */

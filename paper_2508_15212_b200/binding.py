@@ -37,7 +37,11 @@ class spark_params(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("window", ctypes.c_int32), ("keep", ctypes.c_int32),
                 ("page_tokens", ctypes.c_int32), ("dtype", ctypes.c_int32), ("token_budget", ctypes.c_int32),
                 ("pool_kernel", ctypes.c_int32), ("qnorm_eps", ctypes.c_float),
-                ("softmax_scale", ctypes.c_float), ("n_pool_pages", ctypes.c_int64)]
+                ("softmax_scale", ctypes.c_float), ("n_pool_pages", ctypes.c_int64),
+                ("flags", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+SPARK_FLAG_OVERLAP_PREVIOUS = 1
 
 
 _lib = None
@@ -92,10 +96,11 @@ def _stream():
 
 
 def make_params(*, batch, n_q_heads, n_kv_heads, window, keep, dtype, n_pool_pages, head_dim=128,
-                page_tokens=16, token_budget=0, pool_kernel=7, qnorm_eps=0.0, softmax_scale=0.0) -> spark_params:
+                page_tokens=16, token_budget=0, pool_kernel=7, qnorm_eps=0.0, softmax_scale=0.0,
+                flags=0) -> spark_params:
     code = dtype if isinstance(dtype, int) else _DTYPE_CODE[dtype]
     return spark_params(batch, n_q_heads, n_kv_heads, head_dim, window, keep, page_tokens, code,
-                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages)
+                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages, flags, 0)
 
 
 # ---- host-only helpers -----------------------------------------------------------------------------

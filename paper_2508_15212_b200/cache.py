@@ -20,7 +20,7 @@ class SparkCache:
     def __init__(self, *, batch: int, n_q_heads: int, n_kv_heads: int, window: int, keep: int, dtype: str,
                  max_tokens: int, device="cuda", block_table: Optional[torch.Tensor] = None,
                  n_pool_pages: Optional[int] = None, token_budget: int = 0, pool_kernel: int = 7,
-                 softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None):
+                 softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None, flags: int = 0):
         self.device = torch.device(device)
         self.dtype = dtype
         self.max_src_tokens = int(max_tokens)
@@ -37,7 +37,7 @@ class SparkCache:
         self.params = B.make_params(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window,
                                     keep=keep, dtype=_TDT[dtype], n_pool_pages=n_pool_pages,
                                     token_budget=token_budget, pool_kernel=pool_kernel,
-                                    softmax_scale=softmax_scale)
+                                    softmax_scale=softmax_scale, flags=flags)
         self.page_bytes = B.spark_page_bytes(self.params)
         assert self.page_bytes > 0
         self.pages = pages if pages is not None else torch.zeros(n_pool_pages * self.page_bytes,
@@ -109,7 +109,7 @@ def permuted_block_table(batch: int, n_kv_heads: int, lens, device, seed: int, s
 
 
 def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int = None, seed_offset: int = 0,
-                        keep_prompts: int = 0):
+                        keep_prompts: int = 0, flags: int = 0):
     """Configuration 4: prompts are generated, evicted to the token budget and pruned ONE AT A TIME (each
     prompt's dense K/V is freed before the next), into one shared page pool; the result is a batch cache
     whose decode step serves all prompts.  Returns (cache, q [B,Hq,D], kept_tokens [B,Hkv,budget], dense)
@@ -119,7 +119,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
     Hq, Hkv, W, S = config["n_q_heads"], config["n_kv_heads"], config["window"], int(config["seq_lens"])
     budget, pool = int(config["token_budget"]), int(config["pool_kernel"])
     batch = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
-                       max_tokens=min(S, budget), device=device)
+                       max_tokens=min(S, budget), device=device, flags=flags)
     blocks = batch.max_blocks
     qs, kept, dense = [], [], []
     for b in range(Bn):

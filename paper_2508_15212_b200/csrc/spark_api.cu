@@ -20,6 +20,7 @@ spark_status spark::check_params(const spark_params* p)
     if (p->n_pool_pages < 1) return SPARK_ERR_BAD_SHAPE;
     if (p->token_budget < 0) return SPARK_ERR_BAD_SHAPE;
     if (!(p->qnorm_eps >= 0.f) || !(p->softmax_scale >= 0.f)) return SPARK_ERR_BAD_SHAPE;
+    if ((p->flags & ~SPARK_FLAG_OVERLAP_PREVIOUS) || p->reserved != 0) return SPARK_ERR_BAD_SHAPE;
     return SPARK_OK;
 }
 

@@ -51,10 +51,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
     int c0, c1;
     cta_range(*C.plan, static_cast<int>(blockIdx.x), c0, c1);
 
+    if (tid == 0) pdl_launch_dependents();
     if (warp == kConsumerWarps) {
         producer_loop(A, C, ring, c0, c1, lane);
         return;
     }
+    pdl_dependency_wait();                                 // q, qnorm, out and the workspace from here on
     write_empty_sequences<kConsumerThreads>(A, prefix, tid);
 
     float* pscr = pscr_all + warp * 32 * GPP;
@@ -234,8 +236,8 @@ static spark_status launch_f32(const DecodeArgs& A0, int n_sms, int smem_optin, 
                              static_cast<int>(smem)) != cudaSuccess)
         return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
-    decode_f32_kernel<G><<<grid, kDecodeThreads, smem, stream>>>(A);
-    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    return launch_decode_kernel(decode_f32_kernel<G>, grid, kDecodeThreads, smem, stream, A) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 spark_status launch_decode_f32(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream)
@@ -278,6 +280,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.tickets = reinterpret_cast<int*>(ws + kWorkspaceHeader);
     A.partials = reinterpret_cast<float*>(ws + kWorkspaceHeader + align_up(units * sizeof(int), 256));
     A.nslots = 0; A.slot_stride = 0; A.pps = 1;
+    A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
     const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, n_sms, smem_optin, stream)
                                                     : launch_decode_f32(G, A, n_sms, smem_optin, stream);
     if (st == SPARK_OK) ++*launches;

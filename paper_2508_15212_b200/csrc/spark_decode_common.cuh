@@ -39,6 +39,7 @@ struct DecodeArgs {
     int nslots;
     int slot_stride;
     int pps;                                 // pages per step (= per ring slot): 1 or 2
+    int overlap;                             // launched as a programmatic dependent of the preceding kernel
 };
 
 // control block at the start of dynamic shared memory
@@ -127,6 +128,30 @@ __device__ __forceinline__ bool slot_wait(uint64_t* full, volatile int* seq, int
     }
     return mbar_wait(&full[slot], round & 1, abort_flag, status);
 }
+// Programmatic dependent launch (sm_90+).  launch_dependents: the kernel enqueued after this one may be
+// scheduled as CTAs of this grid exit.  dependency_wait: returns once the kernel enqueued before this
+// one has completed and its writes are visible (a no-op for an ordinary launch).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch helper: ordinary launch, or with the programmatic-stream-serialization attribute.
+template <typename Kernel>
+inline cudaError_t launch_decode_kernel(Kernel kernel, int grid, int threads, size_t smem, cudaStream_t stream,
+                                        const DecodeArgs& A)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = A.overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, A);
+}
+
 template <int NT> __device__ __forceinline__ void consumer_sync()
 {
     asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");

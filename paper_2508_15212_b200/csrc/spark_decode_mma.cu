@@ -171,10 +171,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
 #else
 #define SPARK_PROBE() do { } while (0)
 #endif
+    if (tid == 0) pdl_launch_dependents();
     if (warp == kNW) {
         producer_loop(A, C, ring, c0, c1, lane);
         return;
     }
+    pdl_dependency_wait();                                 // q, qnorm, out and the workspace from here on
     write_empty_sequences<kNT>(A, prefix, tid);
 
     const int c = lane & 3, r = lane >> 2;                 // quad lane / fragment row
@@ -424,8 +426,8 @@ static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin,
                              static_cast<int>(smem)) != cudaSuccess)
         return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
-    decode_bf16_kernel<G><<<grid, kThreads, smem, stream>>>(A);
-    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    return launch_decode_kernel(decode_bf16_kernel<G>, grid, kThreads, smem, stream, A) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 spark_status launch_decode_bf16(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream)

@@ -221,3 +221,20 @@ def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
         assert cache.status() == 0
         d = float(np.abs(out.cpu().numpy() - out_ref).max())
         assert d <= TOL[dtype], f"max|delta| {d:.3e}"
+
+
+def test_overlap_flag_gives_identical_results_back_to_back():
+    """Programmatic dependent launch: same workspace, consecutive steps, bitwise the same output."""
+    wl = make("bf16", 2, 16, 4, [4000, 1500], 16, 64, seed=140, gap=False)
+    outs = []
+    for flags in (0, B.SPARK_FLAG_OVERLAP_PREVIOUS):
+        cache = SparkCache(batch=2, n_q_heads=16, n_kv_heads=4, window=16, keep=64, dtype="bf16", max_tokens=4000,
+                           flags=flags)
+        cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+        o = [cache.decode(wl.q) for _ in range(6)]             # launched back to back on one stream
+        assert cache.status() == 0
+        assert all(torch.equal(o[0], x) for x in o[1:])
+        outs.append(o[0])
+    assert torch.equal(outs[0], outs[1])
+    with pytest.raises(B.SparkError):
+        SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype="bf16", max_tokens=64, flags=6)
