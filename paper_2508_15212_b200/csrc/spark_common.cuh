@@ -19,9 +19,11 @@ constexpr int kWorkspaceHeader = 256;
 
 // Byte layout of one page (16 tokens of one KV head).  Private to the library.
 //
-//   vals : T rows of 16 elements.  Row s holds kept slot s of every token (token p at element p); slot s
-//          of a token is its s-th kept channel in ascending channel order.  Rows are 32 bytes (bf16) or
-//          64 bytes (fp32), so the section is exactly T elements per token.
+//   vals : T rows of 16 elements.  Row s holds kept slot s of every token; slot s of a token is its
+//          s-th kept channel in ascending channel order.  Rows are 32 bytes (bf16) or 64 bytes (fp32), so
+//          the section is exactly T elements per token.  In fp32 rows token p sits at element p; in bf16
+//          rows at element (p & 7) * 2 + (p >> 3), so the eight tokens that one half of a matrix
+//          fragment reads together fall into eight different 4-byte banks.
 //   mask : [16][4] uint32, bit (j % 32) of word (j / 32) set <=> channel j kept
 //   mu   : [16] float, mean saliency of the pruned channels
 //   v    : [16][128] elements, dense value rows.  In bf16 pages the 16-byte chunks of row p are stored
@@ -51,7 +53,7 @@ __host__ __device__ inline PageLayout make_layout(int dtype, int keep)
 // byte offset of kept slot s of token p inside the vals section
 __host__ __device__ inline int val_offset(int esize, int p, int s)
 {
-    return (s * kPageTokens + p) * esize;
+    return esize == 2 ? (s * kPageTokens + ((p & 7) * 2 + (p >> 3))) * 2 : (s * kPageTokens + p) * 4;
 }
 
 // byte offset (inside the v section) of the 16-byte chunk c of token p's value row
