@@ -144,6 +144,26 @@ spark_status spark_compress(const spark_params *p,
                             void *workspace, size_t workspace_bytes, spark_stream_t stream);
 
 /*
+ * spark_append -- decode-time append of one token per sequence (Sec. "Preliminaries": the new key and
+ * value are concatenated to the cache, K <- Cat[K, k]).  The paper prunes during prefill and does not say
+ * how keys appended later are treated; here the new key is pruned at once with the sequence's prefill
+ * statistics: w[j] = qnorm[j] * |k[j]|, the `keep` largest channels are kept, mu is the mean of the rest --
+ * exactly what spark_compress would have stored for that token given the same window queries.
+ *
+ *   k_new, v_new   [B][Hkv][D] contiguous, dtype as the cache, 16-byte aligned
+ *   pages, block_table, max_blocks, qnorm   as used by spark_compress / spark_decode_attn; the page that
+ *                  holds token index packed_lens[b] must be listed in the block table (a fresh page is
+ *                  cleared by this call)
+ *   packed_lens    IN/OUT [B]: every sequence with room (packed_lens[b] < 16 * max_blocks) grows by one;
+ *                  a full sequence is left unchanged and SPARK_ERR_DEVICE_BOUNDS is recorded
+ *   workspace      at least 256 bytes, 256-byte aligned (status word only)
+ */
+spark_status spark_append(const spark_params *p, const void *k_new, const void *v_new,
+                          void *pages, const int32_t *block_table, int32_t max_blocks,
+                          const float *qnorm, int32_t *packed_lens,
+                          void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
  * spark_decode_attn -- one decode step over the packed cache (Sec. "Channel Recovery"
  * with the degenerate distribution, then the attention of Sec. "Preliminaries").
  *

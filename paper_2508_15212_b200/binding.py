@@ -22,7 +22,7 @@ SPARK_F32, SPARK_BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
-           "spark_compress", "spark_decode_attn", "spark_decode_attn_noalloc", "spark_unpack_pages",
+           "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_noalloc", "spark_unpack_pages",
            "spark_read_status"]
 
 
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.spark_workspace_init.argtypes = [vp, sz, vp]
         L.spark_compress.restype = i32
         L.spark_compress.argtypes = [P, vp, vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.spark_append.restype = i32
+        L.spark_append.argtypes = [P, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.spark_decode_attn.restype = i32
         L.spark_decode_attn.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.spark_decode_attn_noalloc.restype = i32
@@ -146,6 +148,14 @@ def spark_compress(p: spark_params, q_win, k, v, seq_lens, max_seq_tokens, pages
                                 _ptr(qnorm), _ptr(packed_lens), _ptr(kept_tokens), _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _stream()),
            "spark_compress")
+
+
+def spark_append(p: spark_params, k_new, v_new, pages, block_table, qnorm, packed_lens, workspace) -> None:
+    assert k_new.is_contiguous() and v_new.is_contiguous()
+    _check(lib().spark_append(ctypes.byref(p), _ptr(k_new), _ptr(v_new), _ptr(pages), _ptr(block_table),
+                              block_table.shape[-1], _ptr(qnorm), _ptr(packed_lens), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _stream()),
+           "spark_append")
 
 
 def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse, workspace) -> None:

@@ -57,6 +57,11 @@ class SparkCache:
         B.spark_compress(self.params, q_win, k, v, seq_lens, self.max_src_tokens, self.pages, self.block_table,
                          self.qnorm, self.packed_lens, self.kept_tokens, self.ws_compress)
 
+    def append(self, k_new, v_new) -> None:
+        """One new token per sequence ([B, Hkv, D]), pruned with the prefill statistics."""
+        B.spark_append(self.params, k_new, v_new, self.pages, self.block_table, self.qnorm, self.packed_lens,
+                       self.ws_compress)
+
     def decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
         p = self.params
         if out is None:

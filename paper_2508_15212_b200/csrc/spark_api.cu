@@ -111,6 +111,25 @@ spark_status spark_compress(const spark_params* p, const void* q_win, const void
     return st;
 }
 
+spark_status spark_append(const spark_params* p, const void* k_new, const void* v_new, void* pages,
+                          const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                          int32_t* packed_lens, void* workspace, size_t workspace_bytes, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!k_new || !v_new || !pages || !block_table || !qnorm || !packed_lens || !workspace) return SPARK_ERR_NULL;
+    if (max_blocks < 1) return SPARK_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(pages) & 15) || (reinterpret_cast<uintptr_t>(k_new) & 15) ||
+        (reinterpret_cast<uintptr_t>(v_new) & 15))
+        return SPARK_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < kWorkspaceHeader) return SPARK_ERR_WORKSPACE;
+    int launches = 0;
+    st = launch_append(*p, k_new, v_new, pages, block_table, max_blocks, qnorm, packed_lens, workspace,
+                       static_cast<cudaStream_t>(stream), &launches);
+    if (st == SPARK_OK) g_last_launches = launches;
+    return st;
+}
+
 spark_status spark_decode_attn(const spark_params* p, const void* q, const void* pages,
                                const int32_t* block_table, int32_t max_blocks,
                                const int32_t* packed_lens, const float* qnorm, float* out, float* lse,

@@ -105,6 +105,10 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
                            const float* qnorm, float* out, float* lse, void* workspace,
                            size_t workspace_bytes, cudaStream_t stream, int* launches);
 
+spark_status launch_append(const spark_params& p, const void* k_new, const void* v_new, void* pages,
+                           const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                           int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches);
+
 size_t decode_workspace_bytes(const spark_params& p);
 size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens);
 spark_status launch_evict(const spark_params& p, const void* q_win, const void* k, int64_t sb, int64_t sh,

@@ -52,6 +52,100 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 }
 
 // ------------------------------------------------------------------------------------------------
+// One token of one KV head, one warp: saliency, exact top-T selection, and the token's entries of a
+// page image at `image` (kept values in slot order, mask words, mu).  A lane owns channels
+// 4*lane .. 4*lane+3: `kf` are its key values, `raw` their stored bit patterns, `a` its qnorm entries.
+//
+// Selection is exact: the saliency is one __fmul_rn, its bit pattern (non-negative float) is an
+// order-preserving 31-bit key, the T-th largest key is found by a bitwise radix descent with warp
+// reductions, and keys equal to it are admitted in ascending channel order until T channels are kept.
+// ------------------------------------------------------------------------------------------------
+template <bool kBf16>
+__device__ __forceinline__ void pack_token(unsigned char* image, const PageLayout& L, int p, int T, int lane,
+                                           const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4])
+{
+    const unsigned lt = (1u << lane) - 1u;
+    float w[4];
+    unsigned key[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
+        key[i] = __float_as_uint(w[i]);
+    }
+    // T-th largest key by radix descent over the bits in which the 128 keys differ.  The descent
+    // stops as soon as a candidate threshold has exactly T keys at or above it (then those are the
+    // kept set and no tie can straddle the boundary); otherwise it ends with the exact T-th largest
+    // key and equal keys are admitted in ascending channel order.
+    const unsigned k_or = __reduce_or_sync(kFullMask, key[0] | key[1] | key[2] | key[3]);
+    const unsigned k_and = __reduce_and_sync(kFullMask, key[0] & key[1] & key[2] & key[3]);
+    const unsigned diff = k_or ^ k_and;
+    const int top = diff ? (31 - __clz(diff)) : -1;              // highest bit in which keys differ
+    unsigned thr = (top >= 0) ? (k_and & ~((2u << top) - 1u)) : k_and;   // common leading bits
+    bool exact = false;
+    for (int bit = top; bit >= 0; --bit) {
+        const unsigned cand = thr | (1u << bit);
+        const int mine = (key[0] >= cand) + (key[1] >= cand) + (key[2] >= cand) + (key[3] >= cand);
+        const int cnt = __reduce_add_sync(kFullMask, mine);
+        if (cnt >= T) thr = cand;
+        if (cnt == T) { exact = true; break; }
+    }
+    bool kept[4];
+    if (exact) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kept[i] = key[i] >= thr;
+    } else {
+        unsigned eqb[4];
+        int c_gt = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            c_gt += __popc(__ballot_sync(kFullMask, key[i] > thr));
+            eqb[i] = __ballot_sync(kFullMask, key[i] == thr);
+        }
+        const int need_eq = T - c_gt;
+        int rank = 0;                                        // equal keys on lower channels
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rank += __popc(eqb[i] & lt);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const bool eq = key[i] == thr;
+            kept[i] = key[i] > thr || (eq && rank < need_eq);
+            rank += eq ? 1 : 0;
+        }
+    }
+    // slot of each kept channel = kept channels below it
+    int slot = 0;
+    unsigned nib = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        slot += __popc(__ballot_sync(kFullMask, kept[i]) & lt);
+        nib |= kept[i] ? (1u << i) : 0u;
+    }
+    double pruned = 0.0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (kept[i]) {
+            unsigned char* dst = image + val_offset(L.esize, p, slot);
+            if (kBf16) *reinterpret_cast<unsigned short*>(dst) = static_cast<unsigned short>(raw[i]);
+            else *reinterpret_cast<unsigned*>(dst) = raw[i];
+            ++slot;
+        } else {
+            pruned += static_cast<double>(w[i]);
+        }
+    }
+    unsigned word = nib << (4 * (lane & 7));
+    word |= __shfl_xor_sync(kFullMask, word, 1);
+    word |= __shfl_xor_sync(kFullMask, word, 2);
+    word |= __shfl_xor_sync(kFullMask, word, 4);
+    if ((lane & 7) == 0)
+        reinterpret_cast<unsigned*>(image + L.mask_off)[p * kMaskWords + (lane >> 3)] = word;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
+    if (lane == 0)
+        reinterpret_cast<float*>(image + L.mu_off)[p] =
+            (T < kHeadDim) ? static_cast<float>(pruned / static_cast<double>(kHeadDim - T)) : 0.f;
+}
+
+// ------------------------------------------------------------------------------------------------
 // One CTA builds one page (16 tokens of one KV head) in shared memory and writes it out with
 // coalesced 16-byte stores.  One warp per token, two rounds; a lane owns channels 4*lane .. 4*lane+3.
 //
@@ -96,8 +190,6 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     const float4 a4 = reinterpret_cast<const float4*>(
         A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
-    const unsigned lt = (1u << lane) - 1u;
-
     for (int p = warp; p < kPageTokens; p += 8) {
         const int t = blk * kPageTokens + p;
         if (t >= len) continue;                                   // warp-uniform
@@ -122,84 +214,7 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
             *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) = vv;
         }
-        float w[4];
-        unsigned key[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
-            key[i] = __float_as_uint(w[i]);
-        }
-        // T-th largest key by radix descent over the bits in which the 128 keys differ.  The descent
-        // stops as soon as a candidate threshold has exactly T keys at or above it (then those are the
-        // kept set and no tie can straddle the boundary); otherwise it ends with the exact T-th largest
-        // key and equal keys are admitted in ascending channel order.
-        const unsigned k_or = __reduce_or_sync(kFullMask, key[0] | key[1] | key[2] | key[3]);
-        const unsigned k_and = __reduce_and_sync(kFullMask, key[0] & key[1] & key[2] & key[3]);
-        const unsigned diff = k_or ^ k_and;
-        const int top = diff ? (31 - __clz(diff)) : -1;              // highest bit in which keys differ
-        unsigned thr = (top >= 0) ? (k_and & ~((2u << top) - 1u)) : k_and;   // common leading bits
-        bool exact = false;
-        for (int bit = top; bit >= 0; --bit) {
-            const unsigned cand = thr | (1u << bit);
-            const int mine = (key[0] >= cand) + (key[1] >= cand) + (key[2] >= cand) + (key[3] >= cand);
-            const int cnt = __reduce_add_sync(kFullMask, mine);
-            if (cnt >= T) thr = cand;
-            if (cnt == T) { exact = true; break; }
-        }
-        bool kept[4];
-        if (exact) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) kept[i] = key[i] >= thr;
-        } else {
-            unsigned eqb[4];
-            int c_gt = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                c_gt += __popc(__ballot_sync(kFullMask, key[i] > thr));
-                eqb[i] = __ballot_sync(kFullMask, key[i] == thr);
-            }
-            const int need_eq = T - c_gt;
-            int rank = 0;                                        // equal keys on lower channels
-#pragma unroll
-            for (int i = 0; i < 4; ++i) rank += __popc(eqb[i] & lt);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool eq = key[i] == thr;
-                kept[i] = key[i] > thr || (eq && rank < need_eq);
-                rank += eq ? 1 : 0;
-            }
-        }
-        // slot of each kept channel = kept channels below it
-        int slot = 0;
-        unsigned nib = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            slot += __popc(__ballot_sync(kFullMask, kept[i]) & lt);
-            nib |= kept[i] ? (1u << i) : 0u;
-        }
-        double pruned = 0.0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (kept[i]) {
-                unsigned char* dst = image + val_offset(L.esize, p, slot);
-                if (kBf16) *reinterpret_cast<unsigned short*>(dst) = static_cast<unsigned short>(raw[i]);
-                else *reinterpret_cast<unsigned*>(dst) = raw[i];
-                ++slot;
-            } else {
-                pruned += static_cast<double>(w[i]);
-            }
-        }
-        unsigned word = nib << (4 * (lane & 7));
-        word |= __shfl_xor_sync(kFullMask, word, 1);
-        word |= __shfl_xor_sync(kFullMask, word, 2);
-        word |= __shfl_xor_sync(kFullMask, word, 4);
-        if ((lane & 7) == 0)
-            reinterpret_cast<unsigned*>(image + L.mask_off)[p * kMaskWords + (lane >> 3)] = word;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
-        if (lane == 0)
-            reinterpret_cast<float*>(image + L.mu_off)[p] =
-                (T < kHeadDim) ? static_cast<float>(pruned / static_cast<double>(kHeadDim - T)) : 0.f;
+        pack_token<kBf16>(image, L, p, T, lane, a, kf, raw);
     }
     __syncthreads();
 
@@ -211,6 +226,95 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     uint4* dst = reinterpret_cast<uint4*>(A.pages + static_cast<int64_t>(page_id) * L.page_bytes);
     for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
         dst[i] = reinterpret_cast<const uint4*>(image)[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Decode-time append: one new token per sequence is pruned with the sequence's prefill statistics
+// (qnorm) and written into the next token slot of its last page (a fresh page is zeroed first).
+// One warp per (sequence, KV head); a second one-thread-per-sequence kernel advances packed_lens.
+// ------------------------------------------------------------------------------------------------
+struct AppendArgs {
+    const void* k_new;
+    const void* v_new;
+    unsigned char* pages;
+    const int32_t* block_table;
+    int max_blocks;
+    int B, Hkv, keep;
+    int64_t n_pool_pages;
+    PageLayout L;
+    const float* qnorm;
+    int32_t* packed_lens;
+    int* status;
+};
+
+template <typename E>
+__global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
+{
+    constexpr bool kBf16 = (sizeof(E) == 2);
+    const int h = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+    const PageLayout L = A.L;
+    const int t = A.packed_lens[b];
+    const int blk = t / kPageTokens, p = t - blk * kPageTokens;
+    if (t < 0 || blk >= A.max_blocks) {                       // no room: recorded, nothing written
+        if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    const int page_id = A.block_table[(static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk];
+    if (page_id < 0 || page_id >= A.n_pool_pages) {
+        if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    unsigned char* page = A.pages + static_cast<int64_t>(page_id) * L.page_bytes;
+    if (p == 0) {                                             // first token of a page: clear it
+        for (int i = lane; i < L.page_bytes / 16; i += 32) reinterpret_cast<uint4*>(page)[i] = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+    }
+    const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
+    const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+    const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
+    unsigned raw[4];
+    float kf[4];
+    if (kBf16) {
+        const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.k_new) + row);
+        const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.v_new) + row);
+        raw[0] = kk.x & 0xffffu; raw[1] = kk.x >> 16; raw[2] = kk.y & 0xffffu; raw[3] = kk.y >> 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i] << 16);
+        *reinterpret_cast<uint2*>(page + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) = vv;
+    } else {
+        const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.k_new) + row);
+        const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.v_new) + row);
+        raw[0] = kk.x; raw[1] = kk.y; raw[2] = kk.z; raw[3] = kk.w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
+        *reinterpret_cast<uint4*>(page + L.v_off + v_chunk_offset(4, p, lane)) = vv;
+    }
+    pack_token<kBf16>(page, L, p, A.keep, lane, a, kf, raw);
+}
+
+__global__ void append_advance_kernel(AppendArgs A)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= A.B) return;
+    const int t = A.packed_lens[b];
+    if (t >= 0 && t / kPageTokens < A.max_blocks) A.packed_lens[b] = t + 1;
+}
+
+spark_status launch_append(const spark_params& p, const void* k_new, const void* v_new, void* pages,
+                           const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                           int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches)
+{
+    AppendArgs A;
+    A.k_new = k_new; A.v_new = v_new; A.pages = static_cast<unsigned char*>(pages); A.block_table = block_table;
+    A.max_blocks = max_blocks; A.B = p.batch; A.Hkv = p.n_kv_heads; A.keep = p.keep; A.n_pool_pages = p.n_pool_pages;
+    A.L = make_layout(p.dtype, p.keep); A.qnorm = qnorm; A.packed_lens = packed_lens;
+    A.status = static_cast<int*>(workspace);
+    const dim3 grid(p.n_kv_heads, p.batch);
+    if (p.dtype == SPARK_BF16) append_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(A);
+    else append_token_kernel<float><<<grid, 32, 0, stream>>>(A);
+    append_advance_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(A);
+    *launches += 2;
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -238,3 +238,33 @@ def test_overlap_flag_gives_identical_results_back_to_back():
     assert torch.equal(outs[0], outs[1])
     with pytest.raises(B.SparkError):
         SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype="bf16", max_tokens=64, flags=6)
+
+
+@pytest.mark.parametrize("dtype,keep", [("bf16", 64), ("bf16", 25), ("f32", 38)])
+def test_append_tokens_equals_compressing_the_longer_sequence(dtype, keep):
+    """Prefill S0 tokens, append n more one at a time: the cache must equal what pruning all S0 + n
+    tokens with the same window queries gives (oracle), and the decode output must match."""
+    lens0, n_app = [37, 530, 16], 21
+    full = make(dtype, 3, 8, 2, [l + n_app for l in lens0], 8, keep, seed=150, sigma=1.0 if dtype == "bf16" else 0.5)
+    S = max(lens0) + n_app
+    cache = SparkCache(batch=3, n_q_heads=8, n_kv_heads=2, window=8, keep=keep, dtype=dtype, max_tokens=S)
+    lens0_t = torch.tensor(lens0, dtype=torch.int32, device="cuda")
+    cache.compress(full.q_win, full.k, full.v, lens0_t)                  # prefill sees the first S0 tokens only
+    for i in range(n_app):
+        idx = (lens0_t.long() + i).view(3, 1, 1, 1).expand(3, 2, 1, 128)
+        cache.append(full.k.gather(2, idx).squeeze(2).contiguous(), full.v.gather(2, idx).squeeze(2).contiguous())
+    assert cache.status() == 0
+    assert cache.packed_lens.cpu().tolist() == [l + n_app for l in lens0]
+    wl_cpu = full.to("cpu")
+    a, c, o_ref, _ = oracle_side(wl_cpu, keep)
+    u = cache.unpack()
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c["mask"])
+    assert np.allclose(u["mu"].cpu().numpy(), c["mu"], rtol=1e-6, atol=0)
+    out = cache.decode(full.q)
+    assert float(np.abs(out.cpu().numpy() - o_ref).max()) <= TOL[dtype]
+    # a full sequence is left unchanged and the condition is recorded
+    small = SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=8, keep=keep, dtype=dtype, max_tokens=16)
+    one = make(dtype, 1, 4, 1, [16], 8, keep, seed=151, gap=False)
+    small.compress(one.q_win, one.k, one.v, one.seq_lens)
+    small.append(one.k[:, :, 0].contiguous(), one.v[:, :, 0].contiguous())
+    assert small.packed_lens.cpu().tolist() == [16] and B.spark_read_status(small.ws_compress) == 6
