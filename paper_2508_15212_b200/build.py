@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspark.so")
 SOURCES = ["spark_api.cu", "spark_compress.cu", "spark_decode.cu", "spark_decode_mma.cu",
-           "spark_decode_static.cu", "spark_evict.cu"]
+           "spark_decode_static.cu", "spark_evict.cu", "spark_evict_tc.cu"]
 HEADERS = [os.path.join(CSRC, "spark_common.cuh"), os.path.join(CSRC, "spark_decode_common.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "spark.h")]
 

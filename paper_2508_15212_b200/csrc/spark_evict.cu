@@ -280,6 +280,11 @@ __global__ void __launch_bounds__(1024) evict_select_kernel(EvictArgs A)
     if (tid == 0 && s_base_kept != k) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
 }
 
+bool evict_tc_supported(const spark_params& p);
+spark_status launch_evict_votes_tc(const spark_params& p, const void* q_win, const void* k, int64_t sb, int64_t sh,
+                                   int64_t st, const int32_t* seq_lens, int32_t max_seq_tokens, float* partial,
+                                   float* rowstat, float* votes, int* status, cudaStream_t stream, int* launches);
+
 size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens)
 {
     if (p.token_budget <= 0) return 0;
@@ -311,7 +316,11 @@ spark_status launch_evict(const spark_params& p, const void* q_win, const void* 
     const size_t smem = (static_cast<size_t>(kEvTile + kEvRows) * kEvStride + kEvTile) * sizeof(float);
     const dim3 grid(A.n_tiles, p.n_kv_heads, p.batch), ugrid(p.n_kv_heads, p.batch);
     const bool bf16 = p.dtype == SPARK_BF16;
-    if (A.n_tiles > 0 && max_seq_tokens > p.token_budget) {
+    if (A.n_tiles > 0 && max_seq_tokens > p.token_budget && evict_tc_supported(p)) {
+        const spark_status st_tc = launch_evict_votes_tc(p, q_win, k, sb, sh, st, seq_lens, max_seq_tokens, A.partial,
+                                                         A.rowstat, A.votes, A.status, stream, launches);
+        if (st_tc != SPARK_OK) return st_tc;
+    } else if (A.n_tiles > 0 && max_seq_tokens > p.token_budget) {
         cudaError_t e1 = bf16 ? cudaFuncSetAttribute(evict_scores_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))
                               : cudaFuncSetAttribute(evict_scores_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         cudaError_t e2 = bf16 ? cudaFuncSetAttribute(evict_scores_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))
