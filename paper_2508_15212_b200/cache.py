@@ -127,6 +127,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
                        max_tokens=min(S, budget), device=device, flags=flags)
     blocks = batch.max_blocks
     qs, kept, dense = [], [], []
+    batch.prep_us = []                     # evict + prune time of each prompt (CUDA events)
     for b in range(Bn):
         wl = inputs.make_workload(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=S, window=W,
                                   dtype=config["dtype"], sigma_s=config["sigma_s"],
@@ -136,7 +137,12 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
                          block_table=batch.block_table[b:b + 1].contiguous(),
                          n_pool_pages=batch.params.n_pool_pages, pages=batch.pages)
         assert one.block_table.shape[-1] == blocks
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         one.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+        e1.record()
+        e1.synchronize()
+        batch.prep_us.append(e0.elapsed_time(e1) * 1e3)
         batch.qnorm[b].copy_(one.qnorm[0])
         batch.packed_lens[b:b + 1].copy_(one.packed_lens)
         qs.append(wl.q[0])

@@ -34,6 +34,7 @@ struct EvictArgs {
     float* partial;      // [units][R][n_tiles][2]
     float* rowstat;      // [units][R][2]
     float* votes;        // [units][S_max]
+    unsigned* pooled;    // [units][S_max] pooled votes as order-preserving keys
     int32_t* kept;       // [units][budget]
     int32_t* packed_lens;
     int* status;
@@ -179,7 +180,24 @@ __global__ void evict_rowstats_kernel(EvictArgs A)
     }
 }
 
-// One CTA per unit: pooled votes, exact top-k, ordered compaction.
+// pooled[t] = max of the votes within (pool-1)/2 positions of t (clamped to the prefix), stored as the
+// float's bit pattern: votes are >= 0, so unsigned comparison of the patterns is the order of the values.
+__global__ void __launch_bounds__(256) evict_pool_kernel(EvictArgs A)
+{
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int S = min(A.seq_lens[b], A.S_max);
+    if (S <= A.budget) return;
+    const int P = S - A.W, half = (A.pool - 1) / 2;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= P) return;
+    const int64_t base = static_cast<int64_t>(b * A.Hkv + h) * A.S_max;
+    float m = A.votes[base + t];
+    for (int u = t - half; u <= t + half; ++u)
+        if (u >= 0 && u < P) m = fmaxf(m, A.votes[base + u]);
+    A.pooled[base + t] = __float_as_uint(m);
+}
+
+// One CTA per unit: exact top-k of the pooled votes, ordered compaction.
 __global__ void __launch_bounds__(1024) evict_select_kernel(EvictArgs A)
 {
     __shared__ int hist[256];
@@ -200,14 +218,9 @@ __global__ void __launch_bounds__(1024) evict_select_kernel(EvictArgs A)
         for (int t = tid; t < A.budget; t += blockDim.x) kept[t] = t < S ? t : -1;
         return;
     }
-    const int P = S - A.W, half = (A.pool - 1) / 2, k = A.budget - A.W;
-    const float* votes = A.votes + static_cast<int64_t>(unit) * A.S_max;
-    auto pooled_key = [&](int t) -> unsigned {
-        float m = votes[t];
-        for (int u = t - half; u <= t + half; ++u)
-            if (u >= 0 && u < P) m = fmaxf(m, votes[u]);
-        return __float_as_uint(m);                          // votes are >= 0: the bit pattern keeps the order
-    };
+    const int P = S - A.W, k = A.budget - A.W;
+    const unsigned* pooled = A.pooled + static_cast<int64_t>(unit) * A.S_max;
+    auto pooled_key = [&](int t) -> unsigned { return pooled[t]; };
     // radix select of the k-th largest key, 8 bits per pass
     if (tid == 0) { s_prefix = 0; s_mask = 0; s_need = k; }
     __syncthreads();
@@ -215,9 +228,17 @@ __global__ void __launch_bounds__(1024) evict_select_kernel(EvictArgs A)
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
         const unsigned prefix = s_prefix, mask = s_mask;
-        for (int t = tid; t < P; t += blockDim.x) {
-            const unsigned key = pooled_key(t);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        for (int t0 = 0; t0 < P; t0 += blockDim.x) {        // all lanes iterate together (warp votes below)
+            const int t = t0 + tid;
+            const unsigned key = t < P ? pooled_key(t) : 0u;
+            const bool in = t < P && (key & mask) == prefix;
+            const unsigned bin = (key >> shift) & 255u;
+            // lanes that hit the same bin add once: keys of neighbouring tokens mostly share their top bytes
+            const unsigned active = __ballot_sync(0xffffffffu, in);
+            if (in) {
+                const unsigned peers = __match_any_sync(active, bin);
+                if (lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+            }
         }
         __syncthreads();
         if (tid == 0) {
@@ -293,7 +314,7 @@ size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens)
     const size_t tiles = (max_seq_tokens + kEvTile - 1) / kEvTile;
     size_t bytes = units * R * tiles * 2 * sizeof(float);
     bytes += units * R * 2 * sizeof(float);
-    bytes += units * static_cast<size_t>(max_seq_tokens) * sizeof(float);
+    bytes += 2 * units * static_cast<size_t>(max_seq_tokens) * sizeof(float);      // votes, pooled keys
     return (bytes + 255) / 256 * 256;
 }
 
@@ -312,6 +333,7 @@ spark_status launch_evict(const spark_params& p, const void* q_win, const void* 
     A.partial = reinterpret_cast<float*>(ws + kWorkspaceHeader);
     A.rowstat = A.partial + units * R * A.n_tiles * 2;
     A.votes = A.rowstat + units * R * 2;
+    A.pooled = reinterpret_cast<unsigned*>(A.votes + units * static_cast<size_t>(max_seq_tokens));
     A.kept = kept_tokens; A.packed_lens = packed_lens;
     const size_t smem = (static_cast<size_t>(kEvTile + kEvRows) * kEvStride + kEvTile) * sizeof(float);
     const dim3 grid(A.n_tiles, p.n_kv_heads, p.batch), ugrid(p.n_kv_heads, p.batch);
@@ -332,6 +354,10 @@ spark_status launch_evict(const spark_params& p, const void* q_win, const void* 
         if (bf16) evict_scores_kernel<__nv_bfloat16, 2><<<grid, kEvThreads, smem, stream>>>(A);
         else evict_scores_kernel<float, 2><<<grid, kEvThreads, smem, stream>>>(A);
         *launches += 3;
+    }
+    if (max_seq_tokens > p.token_budget) {
+        evict_pool_kernel<<<dim3((max_seq_tokens + 255) / 256, p.n_kv_heads, p.batch), 256, 0, stream>>>(A);
+        ++*launches;
     }
     evict_select_kernel<<<ugrid, 1024, 0, stream>>>(A);
     ++*launches;

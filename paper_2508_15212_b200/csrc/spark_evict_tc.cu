@@ -63,6 +63,13 @@ __device__ __forceinline__ void tc_mma(unsigned d_tmem, uint64_t a_desc, uint64_
         : "memory");
 }
 
+__device__ __forceinline__ float tc_ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32])
 {
     unsigned r[32];
@@ -113,7 +120,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
     const int tile0 = part * A.tiles_per_cta;
     const int n_tiles_total = (S + kTcTile - 1) / kTcTile;
     const int tile1 = min(n_tiles_total, tile0 + A.tiles_per_cta);
-    const float scale = rsqrtf(static_cast<float>(kHeadDim));
+    // scores are kept in the log2 domain: 2^(s * log2 e) = e^s, one ex2 per probability
+    const float scale = rsqrtf(static_cast<float>(kHeadDim)) * 1.4426950408889634f;
 
     // operand tiles start on a 1024-byte boundary (the swizzle atom); the launch reserves the slack
     unsigned char* q_s = tc_smem + ((1024u - (tc_smem_u32(tc_smem) & 1023u)) & 1023u);   // [2][Rpad][128 B]
@@ -209,8 +217,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
                             const float mn = fmaxf(m, cm);
                             float add = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) add += (v[i] == -INFINITY) ? 0.f : expf(v[i] - mn);
-                            l = l * expf(m - mn) + add;
+                            for (int i = 0; i < 32; ++i) add += tc_ex2(v[i] - mn);          // 2^(-inf) = 0 for masked keys
+                            l = l * tc_ex2(m - mn) + add;
                             m = mn;
                         }
                     }
@@ -226,7 +234,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const int row = c0 + i;
-                        if (row < R) vote += expf(v[i] * scale - row_m[row]) * row_il[row];
+                        if (row < R) vote += tc_ex2(fmaf(v[i], scale, -row_m[row])) * row_il[row];
                     }
                 }
                 if (t < S) A.votes[static_cast<int64_t>(unit) * A.S_max + t] = (t < P) ? vote : 0.f;
@@ -264,7 +272,7 @@ __global__ void evict_rowstats_tc_kernel(EvictTcArgs A, float* rowstat)
             const float m = src[2 * p], l = src[2 * p + 1];
             if (m == -INFINITY) continue;
             const float Mn = fmaxf(M, m);
-            L = L * expf(M - Mn) + l * expf(m - Mn);
+            L = L * exp2f(M - Mn) + l * exp2f(m - Mn);
             M = Mn;
         }
         rowstat[(static_cast<int64_t>(unit) * R + row) * 2] = M;
