@@ -26,6 +26,7 @@ namespace spark {
 constexpr int kNW = 15;                       // consumer warps (+ 1 producer warp = 16 warps, 4 per scheduler)
 constexpr int kNT = kNW * 32;
 constexpr int kThreads = kNT + 32;
+constexpr float kSlack = 8.f;                 // log2 units a score may exceed the running reference maximum
 
 template <int G> struct SmemBf16 {
     static constexpr int kTab = kCtrlBytes + kPrefixBytes;                       // q, q' high, q' low: 3 x [G][128] bf16
@@ -246,6 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
         SPARK_PROBE();      // setup done
 
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float thr[2] = {hv[0] ? -INFINITY : INFINITY, hv[1] ? -INFINITY : INFINITY};
         float o[8][4];
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) { o[mt][0] = 0.f; o[mt][1] = 0.f; o[mt][2] = 0.f; o[mt][3] = 0.f; }
@@ -296,26 +298,50 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                     rk[e] = d2[e] + other;
                 }
                 // ---------------- online softmax over the 16 tokens ----------------
+                // The reference maximum m_run of a head moves only when a score of the page exceeds it
+                // by more than kSlack (log2 units), so most pages skip the warp-wide maximum and the
+                // rescaling; probabilities then lie in (0, 2^kSlack], which fp32 sums and the bf16
+                // high/low split carry without loss.  thr = m_run + kSlack (+inf for unused columns).
                 const float mu[2] = {lds_f32(page + L.mu_off + r * 4), lds_f32(page + L.mu_off + (r + 8) * 4)};
-                float s[2][2], alpha[2], ph[2][2], pl[2][2];
+                float s[2][2];
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
+                for (int e = 0; e < 2; ++e)
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         const float sv = A.scale_log2e * fmaf(mu[j], qsum[e] - rk[2 * j + e], d1[2 * j + e]);
                         s[j][e] = (r + 8 * j < n_valid) ? sv : -INFINITY;
                     }
-                    float mt = fmaxf(s[0][e], s[1][e]);
-                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 4));
-                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 8));
-                    mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 16));
-                    const float m_new = fmaxf(m_run[e], mt);
-                    const float al = ex2(m_run[e] - m_new);
-                    alpha[e] = hv[e] ? al : 1.f;
-                    const float p0 = hv[e] ? ex2(s[0][e] - m_new) : 0.f;
-                    const float p1 = hv[e] ? ex2(s[1][e] - m_new) : 0.f;
-                    l_run[e] = fmaf(l_run[e], alpha[e], p0 + p1);
-                    m_run[e] = m_new;
+                const float over = fmaxf(fmaxf(s[0][0], s[1][0]) - thr[0], fmaxf(s[0][1], s[1][1]) - thr[1]);
+                if (__any_sync(kFull, over > 0.f)) {
+                    float alpha[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float mt = fmaxf(s[0][e], s[1][e]);
+                        mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 4));
+                        mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 8));
+                        mt = fmaxf(mt, __shfl_xor_sync(kFull, mt, 16));
+                        const float m_new = fmaxf(m_run[e], mt);
+                        alpha[e] = hv[e] ? ex2(m_run[e] - m_new) : 1.f;
+                        l_run[e] *= alpha[e];
+                        m_run[e] = m_new;
+                        thr[e] = hv[e] ? m_new + kSlack : INFINITY;
+                    }
+                    float a0 = alpha[0], a1 = alpha[1];      // columns 2c, 2c+1 of every output tile
+                    if (kShared8) {
+                        const float y0 = __shfl_xor_sync(kFull, a0, 2), y1 = __shfl_xor_sync(kFull, a1, 2);
+                        if (c >= 2) { a0 = y0; a1 = y1; }
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < 8; ++mt) {
+                        o[mt][0] *= a0; o[mt][1] *= a1; o[mt][2] *= a0; o[mt][3] *= a1;
+                    }
+                }
+                float ph[2][2], pl[2][2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float p0 = hv[e] ? ex2(s[0][e] - m_run[e]) : 0.f;
+                    const float p1 = hv[e] ? ex2(s[1][e] - m_run[e]) : 0.f;
+                    l_run[e] += p0 + p1;
                     ph[0][e] = bf16_round(p0); pl[0][e] = p0 - ph[0][e];
                     ph[1][e] = bf16_round(p1); pl[1][e] = p1 - ph[1][e];
                 }
@@ -331,20 +357,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                     } else {
                         pb0 = movmatrix_trans(h0); pb1 = movmatrix_trans(h1);
                         pc0 = movmatrix_trans(l0); pc1 = movmatrix_trans(l1);
-                    }
-                }
-                // rescale the running output when a maximum moved (columns 2c, 2c+1 of every tile)
-                {
-                    float a0 = alpha[0], a1 = alpha[1];
-                    if (kShared8) {
-                        const float y0 = __shfl_xor_sync(kFull, a0, 2), y1 = __shfl_xor_sync(kFull, a1, 2);
-                        if (c >= 2) { a0 = y0; a1 = y1; }
-                    }
-                    if (__any_sync(kFull, a0 != 1.0f || a1 != 1.0f)) {
-#pragma unroll
-                        for (int mt = 0; mt < 8; ++mt) {
-                            o[mt][0] *= a0; o[mt][1] *= a1; o[mt][2] *= a0; o[mt][3] *= a1;
-                        }
                     }
                 }
                 // ---------------- P.V: out^T[channel][col] += V^T[channel][token] P^T[token][col] ----------------
