@@ -130,8 +130,21 @@ def compress(k, seq_lens, keep: int, a, *, want_idx=False, want_saliency=False, 
     return out
 
 
+def prune_values(v, seq_lens, keep_v: int):
+    """App. "Pruning Value Cache Channels": per-token top-T_v value channels by magnitude.  -> vmask"""
+    vv, dt = _as_np(v)
+    B, Hkv, S, D = vv.shape
+    sb, sh, st = _kv_strides(vv)
+    lens = _i32(seq_lens)
+    vmask = np.empty((B, Hkv, S, (D + 31) // 32), np.uint32)
+    rc = lib().oracle_prune_values(_ptr(vv), dt, B, Hkv, D, ctypes.c_int64(sb), ctypes.c_int64(sh),
+                                   ctypes.c_int64(st), _ptr(lens), S, int(keep_v), _ptr(vmask))
+    assert rc == 0, rc
+    return vmask
+
+
 def decode_attn(q, k, v, lens, mask, mu, a, *, scale: float = 0.0, path: int = 0,
-                want_scores: bool = False):
+                want_scores: bool = False, vmask=None):
     """Sec. "Channel Recovery" + softmax attention.  -> (out [B,Hq,D] f32, lse [B,Hq] f32[, scores])"""
     qq, dtq = _as_np(q)
     kk, dt = _as_np(k)
@@ -150,11 +163,14 @@ def decode_attn(q, k, v, lens, mask, mu, a, *, scale: float = 0.0, path: int = 0
     out = np.empty((B, Hq, D), np.float32)
     lse = np.empty((B, Hq), np.float32)
     scores = np.zeros((B, Hq, S), np.float64) if want_scores else None
+    if vmask is not None:
+        vmask = np.ascontiguousarray(vmask, dtype=np.uint32)
+        assert vmask.shape == mask.shape
     rc = lib().oracle_decode_attn(_ptr(qq), _ptr(kk), _ptr(vv), dt, B, Hq, Hkv, D,
                                   ctypes.c_int64(sb), ctypes.c_int64(sh), ctypes.c_int64(st),
                                   _ptr(lens), S, _ptr(mask), _ptr(mu), _ptr(a),
                                   ctypes.c_double(scale), int(path), _ptr(out), _ptr(lse),
-                                  _ptr(scores))
+                                  _ptr(scores), _ptr(vmask))
     assert rc == 0, rc
     return (out, lse, scores) if want_scores else (out, lse)
 

@@ -21,6 +21,8 @@
  *   recovery .................. Sec. "Channel Recovery", k~ = w~ / ||q-bar^j||_2,
  *                               degenerate distribution w~ = mu_pruned
  *   attention ................. Sec. "Preliminaries", softmax(q K^T / sqrt(D)) V
+ *   value-channel pruning ..... App. "Pruning Value Cache Channels": per token, the T_v value
+ *                               channels of largest magnitude are kept; the rest are removed
  *
  * Readings taken where the paper is silent (each listed in the design notes):
  *   - ||q-bar^j||_2 of a scalar channel is |q-bar^j|; under GQA the G*W window
@@ -29,7 +31,10 @@
  *   - |q-bar^j| is floored at qnorm_eps before dividing;
  *   - statistics are per token, over that token's pruned channels;
  *   - on equal saliency the lower channel index is kept;
- *   - the 1/sqrt(D) factor scales the whole reconstructed dot product.
+ *   - the 1/sqrt(D) factor scales the whole reconstructed dot product;
+ *   - a pruned value entry contributes nothing to the weighted sum (the appendix says value
+ *     "recovery requires no additional operations"); the importance of a scalar channel is
+ *     its absolute value; ties keep the lower channel.
  *
  * Eviction (observation-window attention-score top-k with max pooling) is not
  * defined by the paper, which only cites the base method and its settings
@@ -178,11 +183,49 @@ int oracle_compress(const void *k, int dtype, int B, int Hkv, int D,
 }
 
 /* ---------------------------------------------------------------------------------
+ * Per-token channel pruning of the values (App. "Pruning Value Cache Channels").
+ *   importance[t][j] = |V[t][j]|
+ *   kept_t  = first T_v channels of (importance descending, j ascending)
+ *   vmask[t] bit (j % 32) of word (j / 32) set  <=>  value channel j kept
+ * v strided like k in oracle_compress.  vmask: [B][Hkv][S_max][MW].  Rows t >= seq_lens[b] are zero.
+ * --------------------------------------------------------------------------------- */
+int oracle_prune_values(const void *v, int dtype, int B, int Hkv, int D,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                        const int32_t *seq_lens, int S_max, int T_v, uint32_t *vmask)
+{
+    if (!v || !seq_lens || !vmask || T_v < 1 || T_v > D) return 1;
+    const int MW = (D + 31) / 32;
+    int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h) {
+            sal_t *row = (sal_t *)malloc(sizeof(sal_t) * (size_t)D);
+            if (!row) { err = 2; continue; }
+            for (int t = 0; t < S_max; ++t) {
+                int64_t u = ((int64_t)b * Hkv + h) * S_max + t;
+                memset(vmask + u * MW, 0, sizeof(uint32_t) * (size_t)MW);
+                if (t >= seq_lens[b]) continue;
+                const int64_t vb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                for (int j = 0; j < D; ++j) {
+                    row[j].w = fabsf((float)load_elem(v, vb + j, dtype));
+                    row[j].j = j;
+                }
+                qsort(row, (size_t)D, sizeof(sal_t), sal_cmp);
+                for (int r = 0; r < T_v; ++r)
+                    vmask[u * MW + row[r].j / 32] |= (uint32_t)1 << (row[r].j % 32);
+            }
+            free(row);
+        }
+    return err;
+}
+
+/* ---------------------------------------------------------------------------------
  * Decode attention with on-the-fly recovery of the pruned key entries.
  *   path 0:  K~[t][j] = K[t][j] if kept else mu[t] / a[j];
  *            s[t] = scale * sum_j q[j] K~[t][j]
  *   path 1:  s[t] = scale * ( sum_{kept} q[j] K[t][j] + mu[t] * sum_{pruned} q[j]/a[j] )
- *   p = softmax_t(s),  out[c] = sum_t p[t] V[t][c],  lse = max + ln sum exp(s - max)
+ *   p = softmax_t(s),  out[c] = sum_t p[t] V^[t][c],  lse = max + ln sum exp(s - max)
+ *   V^[t][c] = V[t][c], or with vmask (optional, value-channel pruning) 0 where channel c of token t is pruned
  * q: [B][Hq][D]; k, v strided as in oracle_compress; lens[b] tokens attended.
  * scale <= 0 selects 1/sqrt(D).  out: [B][Hq][D]; lse (optional): [B][Hq];
  * scores (optional): [B][Hq][S_max] double.  A sequence of length 0 yields zeros / -inf.
@@ -192,7 +235,8 @@ int oracle_decode_attn(const void *q, const void *k, const void *v, int dtype,
                        int64_t stride_b, int64_t stride_h, int64_t stride_t,
                        const int32_t *lens, int S_max,
                        const uint32_t *mask, const float *mu, const float *a,
-                       double scale, int path, float *out, float *lse, double *scores)
+                       double scale, int path, float *out, float *lse, double *scores,
+                       const uint32_t *vmask)
 {
     if (!q || !k || !v || !lens || !mask || !mu || !a || !out || Hkv <= 0 || Hq % Hkv) return 1;
     const int G = Hq / Hkv, MW = (D + 31) / 32;
@@ -243,7 +287,11 @@ int oracle_decode_attn(const void *q, const void *k, const void *v, int dtype,
             for (int t = 0; t < S; ++t) {
                 const double p = exp(s[t] - mx) / den;
                 const int64_t vb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
-                for (int c = 0; c < D; ++c) acc[c] += p * load_elem(v, vb + c, dtype);
+                const uint32_t *vm = vmask ? vmask + (((int64_t)b * Hkv + h) * S_max + t) * MW : NULL;
+                for (int c = 0; c < D; ++c) {
+                    if (vm && !((vm[c / 32] >> (c % 32)) & 1u)) continue;      /* pruned value entry */
+                    acc[c] += p * load_elem(v, vb + c, dtype);
+                }
             }
             for (int c = 0; c < D; ++c) o[c] = (float)acc[c];
             if (lse) lse[(int64_t)b * Hq + i] = (float)(mx + log(den));

@@ -322,3 +322,70 @@ def test_eviction_pool_one_is_plain_top_k_of_causal_window_votes():
     _, _, vote5, pooled5 = oracle.evict(q_win, k, [S], budget=budget, pool=5, want_votes=True)
     for t in range(P):
         assert pooled5[0, 0, t] == vote5[0, 0, max(0, t - 2):min(P, t + 3)].max()
+
+
+# ---------------------------------------------------------------- value-channel pruning (App. "Pruning Value Cache Channels")
+def test_value_pruning_hand_rows_and_ties():
+    # |v| = (3, 1, 0.5, 4, 1, 0, 2, 4): the three largest are channels 3 and 7 (4, tie -> lower first) and 0 (3)
+    v = np.array([3, -1, 0.5, -4, 1, 0, -2, 4], np.float32).reshape(1, 1, 1, 8)
+    assert bits_of(oracle.prune_values(v, [1], 3)[0, 0, 0], 8) == [0, 3, 7]
+    assert bits_of(oracle.prune_values(v, [1], 2)[0, 0, 0], 8) == [3, 7]
+    assert bits_of(oracle.prune_values(v, [1], 1)[0, 0, 0], 8) == [3]          # tie 3 vs 7: lower channel
+    assert bits_of(oracle.prune_values(v, [1], 5)[0, 0, 0], 8) == [0, 1, 3, 6, 7]  # tie 1 vs 4 at |v| = 1
+    assert bits_of(oracle.prune_values(v, [1], 8)[0, 0, 0], 8) == list(range(8))
+
+
+@pytest.mark.parametrize("D,T_v", [(6, 2), (8, 5), (40, 13)])
+def test_value_pruning_maximises_kept_magnitude(D, T_v):
+    """The kept set is the T_v-subset with the largest sum of |v| (brute force for small D, separation beyond)."""
+    rng = np.random.default_rng(11 + D)
+    v = rng.standard_normal((2, 2, 4, D)).astype(np.float32)
+    vm = oracle.prune_values(v, [4, 3], T_v)
+    for b, h, t in itertools.product(range(2), range(2), range(4)):
+        kept = bits_of(vm[b, h, t], D)
+        if t >= [4, 3][b]:
+            assert kept == []
+            continue
+        assert len(kept) == T_v
+        mag = np.abs(v[b, h, t].astype(np.float64))
+        if D <= 8:
+            best = max(itertools.combinations(range(D), T_v), key=lambda c: mag[list(c)].sum())
+            assert kept == list(best)
+        else:
+            assert mag[kept].min() >= np.delete(mag, kept).max()
+
+
+def test_value_pruning_bf16_input_and_full_keep_is_identity():
+    rng = np.random.default_rng(5)
+    q_win, k, v, q = rand_case(rng, B=1, Hq=2, Hkv=1, W=3, D=32, S=9)
+    v16 = (v.view(np.uint32) >> 16).astype(np.uint16)                  # truncated bf16 patterns
+    vf = (v16.astype(np.uint32) << 16).view(np.float32)
+    assert np.array_equal(oracle.prune_values(v16, [9], 7), oracle.prune_values(vf, [9], 7))
+    _, a = oracle.window_mean(q_win, 1)
+    c = oracle.compress(k, [9], 16, a)
+    full = oracle.prune_values(v, [9], 32)
+    assert (full == 0xFFFFFFFF).all()
+    o0, l0 = oracle.decode_attn(q, k, v, [9], c["mask"], c["mu"], a)
+    o1, l1 = oracle.decode_attn(q, k, v, [9], c["mask"], c["mu"], a, vmask=full)
+    assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+
+
+def test_value_pruned_decode_equals_dense_routine_on_zeroed_values():
+    """Pruned value entries contribute nothing: same result as textbook attention over values zeroed by hand,
+    with the scores untouched (the key side is unaffected by the value mask)."""
+    rng = np.random.default_rng(8)
+    q_win, k, v, q = rand_case(rng, B=2, Hq=4, Hkv=2, W=4, D=16, S=11)
+    lens = [11, 6]
+    _, a = oracle.window_mean(q_win, 2)
+    c = oracle.compress(k, lens, 16, a)                                # keys dense -> scores are textbook scores
+    vm = oracle.prune_values(v, lens, 5)
+    out, lse = oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, vmask=vm)
+    for b, i in itertools.product(range(2), range(4)):
+        h, n = i // 2, lens[b]
+        vz = np.zeros((n, 16))
+        for t in range(n):
+            order = sorted(range(16), key=lambda j: (-abs(float(v[b, h, t, j])), j))[:5]
+            vz[t, order] = v[b, h, t, order]
+        ref, ref_lse = dense_attention(q[b, i], k[b, h, :n], vz)
+        assert np.allclose(out[b, i], ref, rtol=0, atol=2e-7)
+        assert abs(lse[b, i] - ref_lse) < 1e-6
