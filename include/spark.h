@@ -23,6 +23,8 @@
  * `page_tokens` consecutive tokens of ONE KV head of one sequence:
  *     kept key values (ascending channel order) | 128-bit channel mask per token
  *     | mu_pruned per token (fp32) | dense value rows
+ * or, with value-channel pruning (keep_v < head_dim), kept value entries and a second
+ * 128-bit mask per token in place of the dense value rows.
  * `block_table[b][h][i]` is the pool index of the page with tokens
  * [16 i, 16 i + 16) of sequence b, KV head h.  The byte layout inside a page is
  * private to the library (spark_page_bytes gives its size; spark_unpack_pages
@@ -69,7 +71,7 @@ typedef struct {
     float   softmax_scale;  /* 0 selects 1/sqrt(head_dim)                                     */
     int64_t n_pool_pages;   /* pages in the pool; every block-table entry must be below it    */
     int32_t flags;          /* bit set of spark_flags (0: none)                               */
-    int32_t reserved;       /* must be 0                                                      */
+    int32_t keep_v;         /* T_v, kept value channels per token; 0 or D: values stay dense   */
 } spark_params;
 
 /* spark_params.flags */
@@ -92,7 +94,8 @@ int32_t spark_keep_count(int32_t head_dim, double ratio);
 size_t spark_page_bytes(const spark_params *p);
 
 /* Bytes the method itself has to read per token and KV head in one decode step:
- * kept values + mask + mu_pruned + dense value row (the roofline numerator).  Host only. */
+ * kept key values + mask + mu_pruned + the dense value row, or with value-channel pruning the
+ * kept value entries + their mask (the roofline numerator).  Host only. */
 size_t spark_algorithmic_bytes_per_token(const spark_params *p);
 
 /* Workspace sizes.  `max_seq_tokens` bounds seq_lens (before eviction).  Either
@@ -116,6 +119,11 @@ spark_status spark_workspace_init(void *workspace, size_t workspace_bytes, spark
  *   mu[t]    = mean of w[t][j] over the pruned channels (0 when keep == head_dim)
  * and the page of token t receives K[t][kept_t] (bit-identical, ascending channel
  * order), the mask, mu[t] and V[t][:].
+ *
+ * With 0 < keep_v < head_dim the value rows are pruned as well (App. "Pruning Value Cache
+ * Channels"): per token the keep_v value channels of largest |V[t][j]| are kept (lower channel
+ * first on ties), bit-identical, in ascending channel order, with their own 128-bit mask; the
+ * other entries are dropped and count as zero in the weighted sum of spark_decode_attn.
  *
  * With token_budget > 0 the tokens are first reduced per KV head to
  * min(S_b, token_budget) by observation-window attention votes (softmax of the
@@ -171,6 +179,7 @@ spark_status spark_append(const spark_params *p, const void *k_new, const void *
  *   K~[t][j] = K[t][j] if channel j of token t was kept, else mu[t] / a[j]
  *   s[t]     = softmax_scale * sum_j q[i][j] * K~[t][j]
  *   out[i]   = sum_t softmax_t(s)[t] * V[t][:]          over t < packed_lens[b]
+ *              (with value-channel pruning, V[t][c] counts as 0 where channel c of token t was dropped)
  * Accumulation is fp32; the softmax is computed online over token splits that are
  * merged by their log-sum-exp.  A sequence of length 0 yields out = 0, lse = -inf.
  *
@@ -220,7 +229,7 @@ spark_status spark_decode_attn_noalloc(const spark_params *p, const void *q,
  *   mask   OUT [B][Hkv][max_tokens][4] uint32, bit (j % 32) of word (j / 32) <=> channel j kept
  *   mu     OUT [B][Hkv][max_tokens] fp32
  *   vals   OUT [B][Hkv][max_tokens][keep] in the cache dtype, ascending channel order
- *   v      OUT [B][Hkv][max_tokens][D] in the cache dtype
+ *   v      OUT [B][Hkv][max_tokens][D] in the cache dtype (dropped value entries read back as 0)
  * Rows t >= packed_lens[b] are written as zeros.
  */
 spark_status spark_unpack_pages(const spark_params *p, const void *pages,
@@ -228,6 +237,14 @@ spark_status spark_unpack_pages(const spark_params *p, const void *pages,
                                 const int32_t *packed_lens, int32_t max_tokens,
                                 uint32_t *mask, float *mu, void *vals, void *v,
                                 spark_stream_t stream);
+
+/* spark_unpack_value_masks -- the per-token value-channel masks (App. "Pruning Value Cache Channels").
+ *   vmask  OUT [B][Hkv][max_tokens][4] uint32, bit (j % 32) of word (j / 32) <=> value channel j kept;
+ *          all ones for live tokens when the values are dense, zeros for rows t >= packed_lens[b]. */
+spark_status spark_unpack_value_masks(const spark_params *p, const void *pages,
+                                      const int32_t *block_table, int32_t max_blocks,
+                                      const int32_t *packed_lens, int32_t max_tokens,
+                                      uint32_t *vmask, spark_stream_t stream);
 
 /* Synchronise `stream` and return the status word of a workspace (SPARK_OK when no
  * kernel recorded an error).  Debug and tests only. */

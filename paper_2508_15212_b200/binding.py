@@ -23,7 +23,7 @@ _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
            "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_noalloc", "spark_unpack_pages",
-           "spark_read_status"]
+           "spark_unpack_value_masks", "spark_read_status"]
 
 
 class SparkError(RuntimeError):
@@ -38,7 +38,7 @@ class spark_params(ctypes.Structure):
                 ("page_tokens", ctypes.c_int32), ("dtype", ctypes.c_int32), ("token_budget", ctypes.c_int32),
                 ("pool_kernel", ctypes.c_int32), ("qnorm_eps", ctypes.c_float),
                 ("softmax_scale", ctypes.c_float), ("n_pool_pages", ctypes.c_int64),
-                ("flags", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("flags", ctypes.c_int32), ("keep_v", ctypes.c_int32)]
 
 
 SPARK_FLAG_OVERLAP_PREVIOUS = 1
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.spark_decode_attn_noalloc.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.spark_unpack_pages.restype = i32
         L.spark_unpack_pages.argtypes = [P, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp]
+        L.spark_unpack_value_masks.restype = i32
+        L.spark_unpack_value_masks.argtypes = [P, vp, vp, i32, vp, i32, vp, vp]
         L.spark_read_status.restype = i32
         L.spark_read_status.argtypes = [vp, vp]
         _lib = L
@@ -99,10 +101,10 @@ def _stream():
 
 def make_params(*, batch, n_q_heads, n_kv_heads, window, keep, dtype, n_pool_pages, head_dim=128,
                 page_tokens=16, token_budget=0, pool_kernel=7, qnorm_eps=0.0, softmax_scale=0.0,
-                flags=0) -> spark_params:
+                flags=0, keep_v=0) -> spark_params:
     code = dtype if isinstance(dtype, int) else _DTYPE_CODE[dtype]
     return spark_params(batch, n_q_heads, n_kv_heads, head_dim, window, keep, page_tokens, code,
-                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages, flags, 0)
+                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages, flags, keep_v)
 
 
 # ---- host-only helpers -----------------------------------------------------------------------------
@@ -179,6 +181,12 @@ def spark_unpack_pages(p: spark_params, pages, block_table, packed_lens, max_tok
                                     _ptr(packed_lens), int(max_tokens), _ptr(mask), _ptr(mu), _ptr(vals),
                                     _ptr(v), _stream()),
            "spark_unpack_pages")
+
+
+def spark_unpack_value_masks(p: spark_params, pages, block_table, packed_lens, max_tokens, vmask) -> None:
+    _check(lib().spark_unpack_value_masks(ctypes.byref(p), _ptr(pages), _ptr(block_table), block_table.shape[-1],
+                                          _ptr(packed_lens), int(max_tokens), _ptr(vmask), _stream()),
+           "spark_unpack_value_masks")
 
 
 def spark_read_status(workspace: torch.Tensor) -> int:

@@ -20,7 +20,8 @@ class SparkCache:
     def __init__(self, *, batch: int, n_q_heads: int, n_kv_heads: int, window: int, keep: int, dtype: str,
                  max_tokens: int, device="cuda", block_table: Optional[torch.Tensor] = None,
                  n_pool_pages: Optional[int] = None, token_budget: int = 0, pool_kernel: int = 7,
-                 softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None, flags: int = 0):
+                 softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None, flags: int = 0,
+                 keep_v: int = 0):
         self.device = torch.device(device)
         self.dtype = dtype
         self.max_src_tokens = int(max_tokens)
@@ -37,7 +38,7 @@ class SparkCache:
         self.params = B.make_params(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window,
                                     keep=keep, dtype=_TDT[dtype], n_pool_pages=n_pool_pages,
                                     token_budget=token_budget, pool_kernel=pool_kernel,
-                                    softmax_scale=softmax_scale, flags=flags)
+                                    softmax_scale=softmax_scale, flags=flags, keep_v=keep_v)
         self.page_bytes = B.spark_page_bytes(self.params)
         assert self.page_bytes > 0
         self.pages = pages if pages is not None else torch.zeros(n_pool_pages * self.page_bytes,
@@ -71,7 +72,7 @@ class SparkCache:
         return out
 
     # -- inspection ------------------------------------------------------------------------------
-    def unpack(self, want_vals=True, want_v=True) -> Dict[str, torch.Tensor]:
+    def unpack(self, want_vals=True, want_v=True, want_vmask=False) -> Dict[str, torch.Tensor]:
         p, n = self.params, self.max_tokens
         tdt = _TDT[self.dtype]
         out = dict(mask=torch.empty(p.batch, p.n_kv_heads, n, 4, dtype=torch.int32, device=self.device),
@@ -82,6 +83,9 @@ class SparkCache:
             out["v"] = torch.empty(p.batch, p.n_kv_heads, n, 128, dtype=tdt, device=self.device)
         B.spark_unpack_pages(p, self.pages, self.block_table, self.packed_lens, n, out["mask"], out["mu"],
                              out.get("vals"), out.get("v"))
+        if want_vmask:
+            out["vmask"] = torch.empty(p.batch, p.n_kv_heads, n, 4, dtype=torch.int32, device=self.device)
+            B.spark_unpack_value_masks(p, self.pages, self.block_table, self.packed_lens, n, out["vmask"])
         return out
 
     def status(self) -> int:

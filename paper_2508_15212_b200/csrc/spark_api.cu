@@ -20,7 +20,8 @@ spark_status spark::check_params(const spark_params* p)
     if (p->n_pool_pages < 1) return SPARK_ERR_BAD_SHAPE;
     if (p->token_budget < 0) return SPARK_ERR_BAD_SHAPE;
     if (!(p->qnorm_eps >= 0.f) || !(p->softmax_scale >= 0.f)) return SPARK_ERR_BAD_SHAPE;
-    if ((p->flags & ~SPARK_FLAG_OVERLAP_PREVIOUS) || p->reserved != 0) return SPARK_ERR_BAD_SHAPE;
+    if (p->flags & ~SPARK_FLAG_OVERLAP_PREVIOUS) return SPARK_ERR_BAD_SHAPE;
+    if (p->keep_v < 0 || p->keep_v > p->head_dim) return SPARK_ERR_BAD_SHAPE;
     return SPARK_OK;
 }
 
@@ -42,14 +43,16 @@ size_t spark_page_bytes(const spark_params* p)
     if (!p || p->head_dim != kHeadDim || p->page_tokens != kPageTokens) return 0;
     if (p->dtype != SPARK_F32 && p->dtype != SPARK_BF16) return 0;
     if (p->keep < 1 || p->keep > kHeadDim) return 0;
-    return static_cast<size_t>(make_layout(p->dtype, p->keep).page_bytes);
+    if (p->keep_v < 0 || p->keep_v > kHeadDim) return 0;
+    return static_cast<size_t>(make_layout(p->dtype, p->keep, p->keep_v).page_bytes);
 }
 
 size_t spark_algorithmic_bytes_per_token(const spark_params* p)
 {
-    if (!p || p->keep < 1 || p->keep > p->head_dim) return 0;
+    if (!p || p->keep < 1 || p->keep > p->head_dim || p->keep_v < 0 || p->keep_v > p->head_dim) return 0;
     const size_t e = (p->dtype == SPARK_BF16) ? 2 : 4;
-    return e * p->keep + 16 + 4 + e * p->head_dim;
+    const int tv = value_keep(p->keep_v);
+    return e * p->keep + 16 + 4 + (tv < kHeadDim ? e * tv + 16 : e * p->head_dim);
 }
 
 spark_status spark_workspace_bytes(const spark_params* p, int64_t max_seq_tokens,
@@ -159,8 +162,22 @@ spark_status spark_unpack_pages(const spark_params* p, const void* pages, const 
     if (max_tokens < 0 || max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
     if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
         return SPARK_ERR_BAD_SHAPE;
-    return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, mask, mu, vals, v,
+    return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, mask, mu, vals, v, nullptr,
                          static_cast<cudaStream_t>(stream));
+}
+
+spark_status spark_unpack_value_masks(const spark_params* p, const void* pages, const int32_t* block_table,
+                                      int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
+                                      uint32_t* vmask, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!pages || !block_table || !packed_lens || !vmask) return SPARK_ERR_NULL;
+    if (max_tokens < 0 || max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
+    if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
+        return SPARK_ERR_BAD_SHAPE;
+    return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, nullptr, nullptr, nullptr,
+                         nullptr, vmask, static_cast<cudaStream_t>(stream));
 }
 
 spark_status spark_read_status(const void* workspace, spark_stream_t stream)

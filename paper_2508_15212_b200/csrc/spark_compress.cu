@@ -4,7 +4,9 @@
 // Method (paper sections): the mean window query replaces per-token queries (Sec. "SparK"); the
 // saliency of channel j of token t is w = |q-bar_j| * |K[t][j]| (Sec. "Problem Formulation"); the T
 // channels of largest w are kept (Eq. (cal)); the mean saliency of the pruned channels is cached per
-// token (App. "Caching Pruned Channel Statistics").
+// token (App. "Caching Pruned Channel Statistics").  With value-channel pruning (App. "Pruning Value
+// Cache Channels") the same per-token selection runs on |V[t][j]| and the page stores the kept values and a
+// second mask instead of the dense value row.
 #include "spark_common.cuh"
 
 namespace spark {
@@ -59,9 +61,14 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 // Selection is exact: the saliency is one __fmul_rn, its bit pattern (non-negative float) is an
 // order-preserving 31-bit key, the T-th largest key is found by a bitwise radix descent with warp
 // reductions, and keys equal to it are admitted in ascending channel order until T channels are kept.
+//
+// The same routine prunes a value row (a = 1, so the key is |V[t][j]| itself): `vals_off` / `mask_off`
+// select the section that receives the kept entries and the mask, and mu is written only when
+// `mu_off` >= 0.
 // ------------------------------------------------------------------------------------------------
 template <bool kBf16>
-__device__ __forceinline__ void pack_token(unsigned char* image, const PageLayout& L, int p, int T, int lane,
+__device__ __forceinline__ void pack_token(unsigned char* image, int esize, int vals_off, int mask_off, int mu_off,
+                                           int p, int T, int lane,
                                            const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4])
 {
     const unsigned lt = (1u << lane) - 1u;
@@ -124,7 +131,7 @@ __device__ __forceinline__ void pack_token(unsigned char* image, const PageLayou
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (kept[i]) {
-            unsigned char* dst = image + val_offset(L.esize, p, slot);
+            unsigned char* dst = image + vals_off + val_offset(esize, p, slot);
             if (kBf16) *reinterpret_cast<unsigned short*>(dst) = static_cast<unsigned short>(raw[i]);
             else *reinterpret_cast<unsigned*>(dst) = raw[i];
             ++slot;
@@ -137,12 +144,55 @@ __device__ __forceinline__ void pack_token(unsigned char* image, const PageLayou
     word |= __shfl_xor_sync(kFullMask, word, 2);
     word |= __shfl_xor_sync(kFullMask, word, 4);
     if ((lane & 7) == 0)
-        reinterpret_cast<unsigned*>(image + L.mask_off)[p * kMaskWords + (lane >> 3)] = word;
+        reinterpret_cast<unsigned*>(image + mask_off)[p * kMaskWords + (lane >> 3)] = word;
+    if (mu_off < 0) return;                                   // warp-uniform
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
     if (lane == 0)
-        reinterpret_cast<float*>(image + L.mu_off)[p] =
+        reinterpret_cast<float*>(image + mu_off)[p] =
             (T < kHeadDim) ? static_cast<float>(pruned / static_cast<double>(kHeadDim - T)) : 0.f;
+}
+
+// Key entries and value entries of one token into the page image (a lane owns channels 4*lane .. 4*lane+3;
+// `kraw` / `vraw` are the stored bit patterns of its key and value entries).
+template <bool kBf16>
+__device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLayout& L, int p, int lane,
+                                              const float (&a)[4], const unsigned (&kraw)[4], const unsigned (&vraw)[4])
+{
+    float kf[4], vf[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        kf[i] = __uint_as_float(kBf16 ? kraw[i] << 16 : kraw[i]);
+        vf[i] = __uint_as_float(kBf16 ? vraw[i] << 16 : vraw[i]);
+    }
+    if (L.keep_v < kHeadDim) {
+        const float one[4] = {1.f, 1.f, 1.f, 1.f};
+        pack_token<kBf16>(image, L.esize, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
+    } else if (kBf16) {
+        *reinterpret_cast<uint2*>(image + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) =
+            make_uint2(vraw[0] | (vraw[1] << 16), vraw[2] | (vraw[3] << 16));
+    } else {
+        *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) =
+            make_uint4(vraw[0], vraw[1], vraw[2], vraw[3]);
+    }
+    pack_token<kBf16>(image, L.esize, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw);
+}
+
+// A lane's four key and value entries of one token row (bit patterns).
+template <bool kBf16>
+__device__ __forceinline__ void load_kv_row(const void* k, const void* v, int64_t row, unsigned (&kraw)[4], unsigned (&vraw)[4])
+{
+    if (kBf16) {
+        const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(k) + row);
+        const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(v) + row);
+        kraw[0] = kk.x & 0xffffu; kraw[1] = kk.x >> 16; kraw[2] = kk.y & 0xffffu; kraw[3] = kk.y >> 16;
+        vraw[0] = vv.x & 0xffffu; vraw[1] = vv.x >> 16; vraw[2] = vv.y & 0xffffu; vraw[3] = vv.y >> 16;
+    } else {
+        const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(k) + row);
+        const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(v) + row);
+        kraw[0] = kk.x; kraw[1] = kk.y; kraw[2] = kk.z; kraw[3] = kk.w;
+        vraw[0] = vv.x; vraw[1] = vv.y; vraw[2] = vv.z; vraw[3] = vv.w;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -180,7 +230,6 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     if (blk * kPageTokens >= len) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const PageLayout L = A.L;
-    const int T = A.keep;
     constexpr bool kBf16 = (sizeof(E) == 2);
 
     for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
@@ -197,24 +246,9 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
         const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
                             static_cast<int64_t>(src_t) * A.st + lane * 4;
-        unsigned raw[4];
-        float kf[4];
-        if (kBf16) {
-            const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.k) + row);
-            const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.v) + row);
-            raw[0] = kk.x & 0xffffu; raw[1] = kk.x >> 16; raw[2] = kk.y & 0xffffu; raw[3] = kk.y >> 16;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i] << 16);
-            *reinterpret_cast<uint2*>(image + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) = vv;
-        } else {
-            const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.k) + row);
-            const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.v) + row);
-            raw[0] = kk.x; raw[1] = kk.y; raw[2] = kk.z; raw[3] = kk.w;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
-            *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) = vv;
-        }
-        pack_token<kBf16>(image, L, p, T, lane, a, kf, raw);
+        unsigned kraw[4], vraw[4];
+        load_kv_row<kBf16>(A.k, A.v, row, kraw, vraw);
+        pack_token_kv<kBf16>(image, L, p, lane, a, kraw, vraw);
     }
     __syncthreads();
 
@@ -272,24 +306,9 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
     const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
     const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
-    unsigned raw[4];
-    float kf[4];
-    if (kBf16) {
-        const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.k_new) + row);
-        const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(A.v_new) + row);
-        raw[0] = kk.x & 0xffffu; raw[1] = kk.x >> 16; raw[2] = kk.y & 0xffffu; raw[3] = kk.y >> 16;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i] << 16);
-        *reinterpret_cast<uint2*>(page + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) = vv;
-    } else {
-        const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.k_new) + row);
-        const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(A.v_new) + row);
-        raw[0] = kk.x; raw[1] = kk.y; raw[2] = kk.z; raw[3] = kk.w;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(raw[i]);
-        *reinterpret_cast<uint4*>(page + L.v_off + v_chunk_offset(4, p, lane)) = vv;
-    }
-    pack_token<kBf16>(page, L, p, A.keep, lane, a, kf, raw);
+    unsigned kraw[4], vraw[4];
+    load_kv_row<kBf16>(A.k_new, A.v_new, row, kraw, vraw);
+    pack_token_kv<kBf16>(page, L, p, lane, a, kraw, vraw);
 }
 
 __global__ void append_advance_kernel(AppendArgs A)
@@ -307,7 +326,7 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     AppendArgs A;
     A.k_new = k_new; A.v_new = v_new; A.pages = static_cast<unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.B = p.batch; A.Hkv = p.n_kv_heads; A.keep = p.keep; A.n_pool_pages = p.n_pool_pages;
-    A.L = make_layout(p.dtype, p.keep); A.qnorm = qnorm; A.packed_lens = packed_lens;
+    A.L = make_layout(p.dtype, p.keep, p.keep_v); A.qnorm = qnorm; A.packed_lens = packed_lens;
     A.status = static_cast<int*>(workspace);
     const dim3 grid(p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16) append_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(A);
@@ -333,6 +352,7 @@ struct UnpackArgs {
     float* mu;
     void* vals;
     void* v;
+    uint32_t* vmask;
 };
 
 __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
@@ -375,19 +395,34 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
                 static_cast<unsigned*>(A.vals)[o] =
                     live ? *reinterpret_cast<const unsigned*>(page + val_offset(4, p, s)) : 0u;
         }
-    if (A.v)
+    if (A.vmask)                                                  // all ones for dense value rows
+        for (int i = threadIdx.x; i < kPageTokens * kMaskWords; i += blockDim.x) {
+            const int p = i / kMaskWords;
+            if (t0 + p >= A.max_tokens) continue;
+            const bool live = page && t0 + p < len;
+            A.vmask[(row0 + p) * kMaskWords + (i % kMaskWords)] =
+                !live ? 0u : (L.keep_v < kHeadDim ? reinterpret_cast<const unsigned*>(page + L.vmask_off)[i] : 0xffffffffu);
+        }
+    if (A.v)                                                      // pruned value entries read back as zero
         for (int i = threadIdx.x; i < kPageTokens * kHeadDim; i += blockDim.x) {
             const int p = i / kHeadDim, j = i % kHeadDim;
             if (t0 + p >= A.max_tokens) continue;
             const bool live = page && t0 + p < len;
             const int64_t o = (row0 + p) * kHeadDim + j;
-            if (L.esize == 2) {
-                const unsigned char* src = page + L.v_off + v_chunk_offset(2, p, j >> 3) + (j & 7) * 2;
-                static_cast<unsigned short*>(A.v)[o] = live ? *reinterpret_cast<const unsigned short*>(src) : 0;
-            } else {
-                const unsigned char* src = page + L.v_off + v_chunk_offset(4, p, j >> 2) + (j & 3) * 4;
-                static_cast<unsigned*>(A.v)[o] = live ? *reinterpret_cast<const unsigned*>(src) : 0u;
+            const unsigned char* src = nullptr;
+            if (live && L.keep_v < kHeadDim) {
+                const unsigned* vm = reinterpret_cast<const unsigned*>(page + L.vmask_off) + p * kMaskWords;
+                if ((vm[j >> 5] >> (j & 31)) & 1u) {
+                    int slot = __popc(vm[j >> 5] & ((1u << (j & 31)) - 1u));
+                    for (int w = 0; w < (j >> 5); ++w) slot += __popc(vm[w]);
+                    src = page + L.v_off + val_offset(L.esize, p, slot);
+                }
+            } else if (live) {
+                src = L.esize == 2 ? page + L.v_off + v_chunk_offset(2, p, j >> 3) + (j & 7) * 2
+                                   : page + L.v_off + v_chunk_offset(4, p, j >> 2) + (j & 3) * 4;
             }
+            if (L.esize == 2) static_cast<unsigned short*>(A.v)[o] = src ? *reinterpret_cast<const unsigned short*>(src) : 0;
+            else static_cast<unsigned*>(A.v)[o] = src ? *reinterpret_cast<const unsigned*>(src) : 0u;
         }
 }
 
@@ -432,7 +467,7 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
     A.lens = packed_lens; A.gather = evict ? kept_tokens : nullptr; A.gather_stride = evict ? p.token_budget : 0;
     A.qnorm = qnorm; A.pages = static_cast<unsigned char*>(pages);
     A.block_table = block_table; A.max_blocks = max_blocks; A.Hkv = p.n_kv_heads; A.keep = p.keep;
-    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep); A.status = status;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep, p.keep_v); A.status = status;
     const dim3 grid(n_blocks, p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16)
         compress_pages_kernel<__nv_bfloat16><<<grid, 256, A.L.page_bytes, stream>>>(A);
@@ -445,15 +480,15 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
 
 spark_status launch_unpack(const spark_params& p, const void* pages, const int32_t* block_table,
                            int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
-                           uint32_t* mask, float* mu, void* vals, void* v, cudaStream_t stream)
+                           uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, cudaStream_t stream)
 {
     const int n_blocks = (max_tokens + kPageTokens - 1) / kPageTokens;
     if (n_blocks == 0) return SPARK_OK;
     UnpackArgs A;
     A.pages = static_cast<const unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.lens = packed_lens; A.max_tokens = max_tokens; A.Hkv = p.n_kv_heads;
-    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep);
-    A.mask = mask; A.mu = mu; A.vals = vals; A.v = v;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep, p.keep_v);
+    A.mask = mask; A.mu = mu; A.vals = vals; A.v = v; A.vmask = vmask;
     unpack_pages_kernel<<<dim3(n_blocks, p.n_kv_heads, p.batch), 128, 0, stream>>>(A);
     if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
     return SPARK_OK;

@@ -167,9 +167,26 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                 __syncwarp();
                 // ---------------- P.V: lane = channels 4*lane .. 4*lane+3 ----------------
                 for (int t = 0; t < n_valid; ++t) {
-                    const unsigned char* vrow = sbase + (t >> 4) * L.page_bytes + L.v_off + (t & 15) * (kHeadDim * 4);
-                    const float4 r = *reinterpret_cast<const float4*>(vrow + lane * 16);
-                    const float vv[4] = {r.x, r.y, r.z, r.w};
+                    const unsigned char* pg = sbase + (t >> 4) * L.page_bytes;
+                    float vv[4];
+                    if (L.keep_v < kHeadDim) {             // pruned values: this lane's nibble of the value mask
+                        const int p = t & 15, wi = lane >> 3, sh = 4 * (lane & 7);
+                        const uint4 vm = *reinterpret_cast<const uint4*>(pg + L.vmask_off + p * 16);
+                        const unsigned word = wi == 0 ? vm.x : (wi == 1 ? vm.y : (wi == 2 ? vm.z : vm.w));
+                        int slot = __popc(word & ((1u << sh) - 1u)) + (wi > 0 ? __popc(vm.x) : 0) +
+                                   (wi > 1 ? __popc(vm.y) : 0) + (wi > 2 ? __popc(vm.z) : 0);
+                        const unsigned nib = (word >> sh) & 0xfu;
+                        const float* vb = reinterpret_cast<const float*>(pg + L.v_off) + p;    // slot s at vb[16 s]
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const bool on = (nib >> c) & 1u;
+                            vv[c] = on ? vb[kPageTokens * slot] : 0.f;
+                            slot += on ? 1 : 0;
+                        }
+                    } else {
+                        const float4 r = *reinterpret_cast<const float4*>(pg + L.v_off + (t & 15) * (kHeadDim * 4) + lane * 16);
+                        vv[0] = r.x; vv[1] = r.y; vv[2] = r.z; vv[3] = r.w;
+                    }
                     float pv[GPP];
 #pragma unroll
                     for (int c4 = 0; c4 < GPP / 4; ++c4) {
@@ -272,7 +289,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.q = q; A.pages = static_cast<const unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.lens = packed_lens; A.qnorm = qnorm; A.out = out; A.lse = lse;
     A.B = p.batch; A.Hq = p.n_q_heads; A.Hkv = p.n_kv_heads; A.n_pool_pages = p.n_pool_pages;
-    A.L = make_layout(p.dtype, p.keep);
+    A.L = make_layout(p.dtype, p.keep, p.keep_v);
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf(static_cast<float>(p.head_dim));
     A.scale_log2e = scale * 1.4426950408889634f;
     unsigned char* ws = static_cast<unsigned char*>(workspace);

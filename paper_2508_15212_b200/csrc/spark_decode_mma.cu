@@ -19,6 +19,11 @@
 // free) and the probabilities, split in bf16 high and low parts so the product keeps ~16 mantissa
 // bits, are moved from the score layout to the operand layout with a warp matrix transpose.
 // Softmax statistics and all accumulators are fp32.
+//
+// With value-channel pruning (App. "Pruning Value Cache Channels") a page carries kept value entries and
+// a second mask instead of dense value rows; the warp first expands them (same nibble walk, zeros where
+// pruned) into a 4 KB tile of its own in shared memory, in the chunk-swizzled row layout of a dense
+// page, and the third contraction reads that tile.
 #include "spark_decode_common.cuh"
 
 namespace spark {
@@ -28,11 +33,14 @@ constexpr int kNT = kNW * 32;
 constexpr int kThreads = kNT + 32;
 constexpr float kSlack = 8.f;                 // log2 units a score may exceed the running reference maximum
 
-template <int G> struct SmemBf16 {
+constexpr int kVTileBytes = kPageTokens * kHeadDim * 2;                          // dense value rows of one page
+
+template <int G, bool kPV> struct SmemBf16 {
     static constexpr int kTab = kCtrlBytes + kPrefixBytes;                       // q, q' high, q' low: 3 x [G][128] bf16
     static constexpr int kQsum = kTab + 3 * G * kHeadDim * 2;                    // [8] float
     static constexpr int kMerge = kQsum + 32;
-    static constexpr int kRing = (kMerge + merge_bytes(kNW, G) + 127) / 128 * 128;
+    static constexpr int kVTile = (kMerge + merge_bytes(kNW, G) + 127) / 128 * 128;   // per-warp tiles (pruned values)
+    static constexpr int kRing = kVTile + (kPV ? kNW * kVTileBytes : 0);
 };
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -140,10 +148,51 @@ __device__ __forceinline__ void expand_nibble(unsigned w, unsigned b0m, unsigned
         : "r"(w), "r"(b0m), "r"(b1m), "r"(b2m), "r"(b3m));
 }
 
-template <int G>
+// The value-side nibble: kept value entries in dense positions, zero where pruned (see expand_nibble).
+__device__ __forceinline__ void expand_nibble_v(unsigned w, unsigned b0m, unsigned b1m, unsigned b2m, unsigned b3m,
+                                                unsigned& addr, unsigned& k0, unsigned& k1)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p0, p1, p2, p3;\n\t"
+        ".reg .b32 t0, t1, t2, t3;\n\t"
+        ".reg .b16 h0, h1, h2, h3;\n\t"
+        "and.b32 t0, %3, %4;\n\t"
+        "and.b32 t1, %3, %5;\n\t"
+        "and.b32 t2, %3, %6;\n\t"
+        "and.b32 t3, %3, %7;\n\t"
+        "setp.ne.u32 p0, t0, 0;\n\t"
+        "setp.ne.u32 p1, t1, 0;\n\t"
+        "setp.ne.u32 p2, t2, 0;\n\t"
+        "setp.ne.u32 p3, t3, 0;\n\t"
+        "mov.b16 h0, 0;\n\t"
+        "mov.b16 h1, 0;\n\t"
+        "mov.b16 h2, 0;\n\t"
+        "mov.b16 h3, 0;\n\t"
+        "@p0 ld.shared.u16 h0, [%2];\n\t"
+        "@p0 add.u32 %2, %2, 32;\n\t"
+        "@p1 ld.shared.u16 h1, [%2];\n\t"
+        "@p1 add.u32 %2, %2, 32;\n\t"
+        "@p2 ld.shared.u16 h2, [%2];\n\t"
+        "@p2 add.u32 %2, %2, 32;\n\t"
+        "@p3 ld.shared.u16 h3, [%2];\n\t"
+        "@p3 add.u32 %2, %2, 32;\n\t"
+        "mov.b32 %0, {h0, h1};\n\t"
+        "mov.b32 %1, {h2, h3};\n\t"
+        "}"
+        : "=&r"(k0), "=&r"(k1), "+r"(addr)
+        : "r"(w), "r"(b0m), "r"(b1m), "r"(b2m), "r"(b3m));
+}
+
+__device__ __forceinline__ void sts_u32x4(unsigned addr, unsigned a, unsigned b, unsigned c, unsigned d)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+template <int G, bool kPV>
 __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeArgs A)
 {
-    using S = SmemBf16<G>;
+    using S = SmemBf16<G, kPV>;
     constexpr bool kShared8 = (G <= 4);        // q' high and low parts share one 8-column operand
     extern __shared__ __align__(128) unsigned char smem[];
     const Ctrl C = make_ctrl(smem);
@@ -360,8 +409,36 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                     }
                 }
                 // ---------------- P.V: out^T[channel][col] += V^T[channel][token] P^T[token][col] ----------------
+                unsigned vbase = page + L.v_off;
+                if (kPV) {
+                    // lane (r, c) expands mask word c of tokens r and r + 8: channels 32c + 8u .. + 7 of a
+                    // token are one 16-byte chunk, stored at chunk index (4c + u) ^ r of the token's row
+                    vbase = smem_u32(smem + S::kVTile) + warp * kVTileBytes;
+                    unsigned vw[2], va[2];
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        vw[j] = lds_u32(page + L.vmask_off + (8 * j + r) * 16 + c * 4);
+                        const int cnt = __popc(vw[j]);
+                        int x = cnt;
+                        int t = __shfl_up_sync(kFull, x, 1, 4);
+                        if (c >= 1) x += t;
+                        t = __shfl_up_sync(kFull, x, 2, 4);
+                        if (c >= 2) x += t;
+                        va[j] = page + L.v_off + (r * 2 + j) * 2 + (x - cnt) * 32;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            unsigned e0, e1, e2, e3;
+                            expand_nibble_v(vw[j], 1u << (8 * u), 2u << (8 * u), 4u << (8 * u), 8u << (8 * u), va[j], e0, e1);
+                            expand_nibble_v(vw[j], 16u << (8 * u), 32u << (8 * u), 64u << (8 * u), 128u << (8 * u), va[j], e2, e3);
+                            sts_u32x4(vbase + (8 * j + r) * (kHeadDim * 2) + (((4 * c + u) ^ r) << 4), e0, e1, e2, e3);
+                        }
+                    __syncwarp();
+                }
                 const int mi = lane >> 3, rr = lane & 7;
-                const unsigned vrow = page + L.v_off + (((mi >> 1) << 3) + rr) * (kHeadDim * 2);
+                const unsigned vrow = vbase + (((mi >> 1) << 3) + rr) * (kHeadDim * 2);
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) {
                     unsigned a0, a1, a2, a3;
@@ -422,11 +499,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
 #endif
 }
 
-template <int G>
+template <int G, bool kPV>
 static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin, cudaStream_t stream)
 {
     DecodeArgs A = A0;
-    using S = SmemBf16<G>;
+    using S = SmemBf16<G, kPV>;
     A.pps = 1;
     A.slot_stride = static_cast<int>(align_up(static_cast<size_t>(A.L.page_bytes), 128));
     int ns = (smem_optin - S::kRing) / A.slot_stride;
@@ -434,25 +511,26 @@ static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin,
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
     const size_t smem = S::kRing + static_cast<size_t>(ns) * A.slot_stride;
-    if (cudaFuncSetAttribute(decode_bf16_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(decode_bf16_kernel<G, kPV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)
         return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
-    return launch_decode_kernel(decode_bf16_kernel<G>, grid, kThreads, smem, stream, A) == cudaSuccess
+    return launch_decode_kernel(decode_bf16_kernel<G, kPV>, grid, kThreads, smem, stream, A) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 spark_status launch_decode_bf16(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream)
 {
+    const bool pv = A.L.keep_v < kHeadDim;                  // value rows are pruned: expand them per page
     switch (G) {
-        case 1: return launch_bf16<1>(A, n_sms, smem_optin, stream);
-        case 2: return launch_bf16<2>(A, n_sms, smem_optin, stream);
-        case 3: return launch_bf16<3>(A, n_sms, smem_optin, stream);
-        case 4: return launch_bf16<4>(A, n_sms, smem_optin, stream);
-        case 5: return launch_bf16<5>(A, n_sms, smem_optin, stream);
-        case 6: return launch_bf16<6>(A, n_sms, smem_optin, stream);
-        case 7: return launch_bf16<7>(A, n_sms, smem_optin, stream);
-        case 8: return launch_bf16<8>(A, n_sms, smem_optin, stream);
+        case 1: return pv ? launch_bf16<1, true>(A, n_sms, smem_optin, stream) : launch_bf16<1, false>(A, n_sms, smem_optin, stream);
+        case 2: return pv ? launch_bf16<2, true>(A, n_sms, smem_optin, stream) : launch_bf16<2, false>(A, n_sms, smem_optin, stream);
+        case 3: return pv ? launch_bf16<3, true>(A, n_sms, smem_optin, stream) : launch_bf16<3, false>(A, n_sms, smem_optin, stream);
+        case 4: return pv ? launch_bf16<4, true>(A, n_sms, smem_optin, stream) : launch_bf16<4, false>(A, n_sms, smem_optin, stream);
+        case 5: return pv ? launch_bf16<5, true>(A, n_sms, smem_optin, stream) : launch_bf16<5, false>(A, n_sms, smem_optin, stream);
+        case 6: return pv ? launch_bf16<6, true>(A, n_sms, smem_optin, stream) : launch_bf16<6, false>(A, n_sms, smem_optin, stream);
+        case 7: return pv ? launch_bf16<7, true>(A, n_sms, smem_optin, stream) : launch_bf16<7, false>(A, n_sms, smem_optin, stream);
+        case 8: return pv ? launch_bf16<8, true>(A, n_sms, smem_optin, stream) : launch_bf16<8, false>(A, n_sms, smem_optin, stream);
         default: return SPARK_ERR_UNSUPPORTED;
     }
 }

@@ -31,28 +31,36 @@ def to_np(t):
     return t.numpy()
 
 
-def oracle_side(wl_cpu, keep):
+def oracle_side(wl_cpu, keep, keep_v=0):
     Hkv = wl_cpu.k.shape[1]
     _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
     c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a, want_idx=True)
-    out, lse = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a)
+    c["vmask"] = oracle.prune_values(wl_cpu.v, wl_cpu.seq_lens, keep_v) if 0 < keep_v < 128 else None
+    out, lse = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a,
+                                  vmask=c["vmask"])
     return a, c, out, lse
 
 
-def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True):
+def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True, keep_v=0):
     """wl lives on the GPU; returns max|delta| of the attention output."""
     Bn, Hq, Hkv, W, D, S = wl.shape
     wl_cpu = wl.to("cpu")
-    a, c, o_ref, lse_ref = oracle_side(wl_cpu, keep)
+    a, c, o_ref, lse_ref = oracle_side(wl_cpu, keep, keep_v)
     cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
-                       max_tokens=S, block_table=block_table, n_pool_pages=n_pool_pages)
+                       max_tokens=S, block_table=block_table, n_pool_pages=n_pool_pages, keep_v=keep_v)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     lens = wl_cpu.seq_lens.tolist()
     assert cache.packed_lens.cpu().tolist() == lens
     assert np.array_equal(cache.qnorm.cpu().numpy(), a), "qnorm must be bit-exact"
-    u = cache.unpack()
+    u = cache.unpack(want_vmask=True)
     mask = u["mask"].cpu().numpy().view(np.uint32)
     assert np.array_equal(mask, c["mask"]), "kept-channel masks must be bit-exact"
+    vmask = u["vmask"].cpu().numpy().view(np.uint32)
+    if c["vmask"] is not None:
+        assert np.array_equal(vmask, c["vmask"]), "value-channel masks must be bit-exact"
+    else:
+        live = np.arange(S)[None, None, :, None] < np.asarray(lens)[:, None, None, None]
+        assert np.array_equal(vmask, np.where(live, np.uint32(0xFFFFFFFF), np.uint32(0)) + np.zeros_like(vmask))
     mu = u["mu"].cpu().numpy()
     assert np.allclose(mu, c["mu"], rtol=1e-6, atol=0)
     if check_vals:
@@ -63,6 +71,9 @@ def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True):
             want_vals[b, :, n:] = 0
             vv[b, :, n:] = 0
         assert np.array_equal(to_np(u["vals"]), want_vals), "kept values must be bit-identical copies"
+        if c["vmask"] is not None:                                   # dropped value entries read back as zero
+            bits = (c["vmask"][..., None] >> np.arange(32, dtype=np.uint32)) & 1
+            vv = np.where(bits.reshape(vv.shape).astype(bool), vv, np.zeros_like(vv))
         assert np.array_equal(to_np(u["v"]), vv)
     lse = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
     out = cache.decode(wl.q, lse=lse)
@@ -268,3 +279,52 @@ def test_append_tokens_equals_compressing_the_longer_sequence(dtype, keep):
     small.compress(one.q_win, one.k, one.v, one.seq_lens)
     small.append(one.k[:, :, 0].contiguous(), one.v[:, :, 0].contiguous())
     assert small.packed_lens.cpu().tolist() == [16] and B.spark_read_status(small.ws_compress) == 6
+
+
+# ---- value-channel pruning (App. "Pruning Value Cache Channels") ------------------------------------
+@pytest.mark.parametrize("keep,keep_v", [(64, 64), (64, 89), (25, 25), (38, 1), (128, 64), (64, 127)])
+def test_value_pruning_bf16_ragged(keep, keep_v):
+    wl = make("bf16", 3, 8, 2, [1, 37, 530], 8, keep, seed=300 + keep + keep_v)
+    check_case(wl, keep, keep_v=keep_v)
+
+
+@pytest.mark.parametrize("G,keep,keep_v", [(1, 64, 64), (7, 38, 64), (8, 64, 25)])
+def test_value_pruning_group_sizes_and_paged_pool(G, keep, keep_v):
+    lens = [300, 47]
+    wl = make("bf16", 2, 2 * G, 2, lens, 16, keep, seed=340 + G)
+    from paper_2508_15212_b200.cache import permuted_block_table
+    table, n_pages = permuted_block_table(2, 2, lens, "cuda", seed=7, spare=3)
+    check_case(wl, keep, block_table=table, n_pool_pages=n_pages, keep_v=keep_v)
+
+
+def test_value_pruning_fp32_storage():
+    wl = make("f32", 2, 4, 2, [130, 33], 8, 64, seed=360, sigma=0.5)
+    check_case(wl, 64, keep_v=48)
+
+
+def test_value_pruning_llama_32k_half_half():
+    """The (0.5 + 0.5) setting at the 32K shape: several CTAs per unit, last-arriver merge."""
+    wl = inputs.config_workload(1, device="cuda")
+    inputs.enforce_saliency_gap(wl, 64)
+    d = check_case(wl, 64, check_vals=False, keep_v=64)
+    assert d <= 2e-3
+
+
+def test_value_pruning_append_matches_compressing_the_longer_sequence():
+    lens0, extra = [37, 16], 20
+    wl = make("bf16", 2, 8, 2, [n + extra for n in lens0], 8, 64, seed=370)
+    Bn, Hq, Hkv, W, D, S = wl.shape
+    full = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=64, dtype="bf16", max_tokens=S, keep_v=40)
+    full.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    grown = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=64, dtype="bf16", max_tokens=S, keep_v=40)
+    grown.compress(wl.q_win, wl.k, wl.v, torch.tensor(lens0, dtype=torch.int32, device="cuda"))
+    for step in range(extra):
+        idx = torch.tensor([n + step for n in lens0], device="cuda")
+        k_new = wl.k[torch.arange(Bn, device="cuda"), :, idx].contiguous()
+        v_new = wl.v[torch.arange(Bn, device="cuda"), :, idx].contiguous()
+        grown.append(k_new, v_new)
+    assert grown.status() == 0 and grown.packed_lens.cpu().tolist() == wl.seq_lens.cpu().tolist()
+    ua, ub = full.unpack(want_vmask=True), grown.unpack(want_vmask=True)
+    for key in ("mask", "mu", "vals", "v", "vmask"):
+        assert torch.equal(ua[key], ub[key]), key
+    assert torch.equal(full.decode(wl.q), grown.decode(wl.q))
