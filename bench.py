@@ -99,25 +99,28 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def oracle_decode_time(wl_cpu, keep, reps=3):
+def oracle_decode_time(wl_cpu, keep, reps=3, keep_v=0):
     """Times the CPU oracle's decode (window mean and compress are prepared, untimed)."""
     import oracle
     Hkv = wl_cpu.k.shape[1]
     _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
     c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a)
-    oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a)   # warm
+    vm = oracle.prune_values(wl_cpu.v, wl_cpu.seq_lens, keep_v) if 0 < keep_v < 128 else None
+    oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a, vmask=vm)   # warm
     ts = []
     for _ in range(reps):
         t0 = time.perf_counter()
-        out, _ = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a)
+        out, _ = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a, vmask=vm)
         ts.append(time.perf_counter() - t0)
     return statistics.median(ts), oracle.threads(), out
 
 
-def workload_desc(cfg, keep, copies=None):
+def workload_desc(cfg, keep, copies=None, keep_v=0):
     d = {"workload": cfg["name"], "batch": cfg["batch"], "n_q_heads": cfg["n_q_heads"],
          "n_kv_heads": cfg["n_kv_heads"], "head_dim": cfg["head_dim"], "cached_tokens": cfg["seq_lens"],
          "window": cfg["window"], "pruning_ratio": cfg["ratio"], "keep": keep, "page_tokens": 16}
+    if 0 < keep_v < 128:
+        d["value_keep"] = keep_v                     # value-channel pruning on top of the named workload
     if copies is not None:
         d["cold_cache"] = f"rotation over {copies} packed-cache copies (copies*bytes >= 4*L2)"
     return d
@@ -164,6 +167,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--keep", type=int, default=0, help="override the kept-channel count T")
     ap.add_argument("--ratio", type=float, default=None, help="pruning ratio (configuration 5 sweeps 0.3/0.5/0.7/0.8)")
+    ap.add_argument("--ratio-v", type=float, default=None,
+                    help="also prune value channels with this ratio (default: values stay dense)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-overlap", action="store_true",
                     help="ordinary launches (default: each step may start its page stream while the previous drains)")
@@ -180,6 +185,7 @@ def main():
         cfg["batch"] = args.batch
     cfg["ratio"] = ratio
     keep = args.keep or inputs.keep_count(cfg["head_dim"], ratio)
+    keep_v = inputs.keep_count(cfg["head_dim"], args.ratio_v) if args.ratio_v is not None else 0
     if isinstance(cfg["seq_lens"], tuple):
         cfg["seq_lens"] = list(cfg["seq_lens"])
 
@@ -218,11 +224,12 @@ def main():
     if "token_budget" in cfg:          # prompts evicted and pruned one at a time into one batch cache
         per_tok = B.spark_algorithmic_bytes_per_token(B.make_params(
             batch=1, n_q_heads=cfg["n_q_heads"], n_kv_heads=cfg["n_kv_heads"], window=cfg["window"], keep=keep,
-            dtype=torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32, n_pool_pages=1))
+            dtype=torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32, n_pool_pages=1, keep_v=keep_v))
         alg_bytes = per_tok * cfg["n_kv_heads"] * cfg["token_budget"] * cfg["batch"]
         copies = max(1, -(-4 * l2 // alg_bytes))
         for c in range(copies):
-            cache, q, _, _ = build_evicted_batch(cfg, keep, seed_offset=dist_utils.rank_seed_offset(rank, c), flags=flags)
+            cache, q, _, _ = build_evicted_batch(cfg, keep, seed_offset=dist_utils.rank_seed_offset(rank, c), flags=flags,
+                                                     keep_v=keep_v)
             out = torch.empty(cfg["batch"], cfg["n_q_heads"], D, dtype=torch.float32, device="cuda")
             step_sets.append([(cache, q, out)])
             prep = sorted(cache.prep_us)
@@ -236,7 +243,7 @@ def main():
             lens = wl_l.seq_lens.tolist()
             table, n_pages = permuted_block_table(Bn, Hkv, lens, "cuda", seed=977 * layer + rank)
             cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl_l.dtype,
-                               max_tokens=S, block_table=table, n_pool_pages=n_pages, flags=flags)
+                               max_tokens=S, block_table=table, n_pool_pages=n_pages, flags=flags, keep_v=keep_v)
             cache.compress(wl_l.q_win, wl_l.k, wl_l.v, wl_l.seq_lens)
             alg_bytes += cache.algorithmic_bytes_per_token * Hkv * sum(lens)
             layer_set.append((cache, wl_l.q.clone(), torch.empty(Bn, Hq, D, dtype=torch.float32, device="cuda")))
@@ -253,7 +260,7 @@ def main():
         Bn, Hq, Hkv, W, _, S = wl.shape
         lens = wl.seq_lens.tolist()
         mk = lambda: SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
-                                max_tokens=S, flags=flags)
+                                max_tokens=S, flags=flags, keep_v=keep_v)
         first = mk()
         alg_bytes = first.algorithmic_bytes_per_token * Hkv * sum(lens)
         copies = max(1, min(64, -(-4 * l2 // max(alg_bytes, 1))))
@@ -364,7 +371,7 @@ def main():
     cpu_baseline, max_err = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and wl is not None:
         wl_cpu = wl.to("cpu")
-        t_or, cores, o_ref = oracle_decode_time(wl_cpu, keep)
+        t_or, cores, o_ref = oracle_decode_time(wl_cpu, keep, keep_v=keep_v)
         cpu_baseline = {"value": t_or * 1e6, "unit": "us/step", "cores": cores, "kind": "oracle",
                         "sample": "one full decode step of the workload, median of 3"}
         max_err = float((first.decode(wl.q).cpu().numpy() - o_ref).__abs__().max())
@@ -377,7 +384,7 @@ def main():
             "metric": METRIC, "value": us_step, "unit": "us/step", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": us_step / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": cfg["dtype"], "data": "synthetic",
-            "config": dict(workload_desc(cfg, keep, copies),
+            "config": dict(workload_desc(cfg, keep, copies, keep_v),
                            launch=("programmatic dependent launch: the page stream of step i+1 may start while step i "
                                    "drains; q, out and workspace wait for step i" if flags else "ordinary launches")),
             "hbm_gbs": gbs, "hbm_gbs_all_gpus": dist_utils.aggregate_throughput(alg_bytes / 1e9, world, us_step * 1e-6),
@@ -390,7 +397,7 @@ def main():
             "gpu_launches": args.steps * launches_per_step * B.spark_last_launch_count(),
             "launches_per_step": launches_per_step,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                         "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(name),
+                         "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(name) if not keep_v else None,
                          "kernel": "spark::decode_bf16_kernel" if cfg["dtype"] == "bf16" else "spark::decode_f32_kernel",
                          "algorithmic_bytes_per_launch": alg_bytes / launches_per_step,
                          "avg_launch_us": us_step / launches_per_step},

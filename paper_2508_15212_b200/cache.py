@@ -118,7 +118,7 @@ def permuted_block_table(batch: int, n_kv_heads: int, lens, device, seed: int, s
 
 
 def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int = None, seed_offset: int = 0,
-                        keep_prompts: int = 0, flags: int = 0):
+                        keep_prompts: int = 0, flags: int = 0, keep_v: int = 0):
     """Configuration 4: prompts are generated, evicted to the token budget and pruned ONE AT A TIME (each
     prompt's dense K/V is freed before the next), into one shared page pool; the result is a batch cache
     whose decode step serves all prompts.  Returns (cache, q [B,Hq,D], kept_tokens [B,Hkv,budget], dense)
@@ -128,7 +128,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
     Hq, Hkv, W, S = config["n_q_heads"], config["n_kv_heads"], config["window"], int(config["seq_lens"])
     budget, pool = int(config["token_budget"]), int(config["pool_kernel"])
     batch = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
-                       max_tokens=min(S, budget), device=device, flags=flags)
+                       max_tokens=min(S, budget), device=device, flags=flags, keep_v=keep_v)
     blocks = batch.max_blocks
     qs, kept, dense = [], [], []
     batch.prep_us = []                     # evict + prune time of each prompt (CUDA events)
@@ -139,7 +139,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
         one = SparkCache(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
                          max_tokens=S, device=device, token_budget=budget, pool_kernel=pool,
                          block_table=batch.block_table[b:b + 1].contiguous(),
-                         n_pool_pages=batch.params.n_pool_pages, pages=batch.pages)
+                         n_pool_pages=batch.params.n_pool_pages, pages=batch.pages, keep_v=keep_v)
         assert one.block_table.shape[-1] == blocks
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
