@@ -412,7 +412,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                 unsigned vbase = page + L.v_off;
                 if (kPV) {
                     // lane (r, c) expands mask word c of tokens r and r + 8: channels 32c + 8u .. + 7 of a
-                    // token are one 16-byte chunk, stored at chunk index (4c + u) ^ r of the token's row
+                    // token are 16-byte chunk k = 4c + u, stored at chunk index k ^ r ^ ((k >> 3) << 1) of the
+                    // token's row (the extra term keeps the four lanes of a row on different banks)
                     vbase = smem_u32(smem + S::kVTile) + warp * kVTileBytes;
                     unsigned vw[2], va[2];
 #pragma unroll
@@ -433,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                             unsigned e0, e1, e2, e3;
                             expand_nibble_v(vw[j], 1u << (8 * u), 2u << (8 * u), 4u << (8 * u), 8u << (8 * u), va[j], e0, e1);
                             expand_nibble_v(vw[j], 16u << (8 * u), 32u << (8 * u), 64u << (8 * u), 128u << (8 * u), va[j], e2, e3);
-                            sts_u32x4(vbase + (8 * j + r) * (kHeadDim * 2) + (((4 * c + u) ^ r) << 4), e0, e1, e2, e3);
+                            sts_u32x4(vbase + (8 * j + r) * (kHeadDim * 2) + (((4 * c + u) ^ r ^ (c & 2)) << 4), e0, e1, e2, e3);
                         }
                     __syncwarp();
                 }
@@ -442,7 +443,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) {
                     unsigned a0, a1, a2, a3;
-                    ldmatrix_x4_trans(a0, a1, a2, a3, vrow + (((2 * mt + (mi & 1)) ^ rr) << 4));
+                    ldmatrix_x4_trans(a0, a1, a2, a3, vrow + (((2 * mt + (mi & 1)) ^ rr ^ (kPV ? ((mt >> 2) << 1) : 0)) << 4));
                     mma_bf16(o[mt], a0, a1, a2, a3, pb0, pb1);
                     if (!kShared8) mma_bf16(o[mt], a0, a1, a2, a3, pc0, pc1);
                 }
