@@ -31,7 +31,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the ncu capture summarised in
 # profiles/ (bytes); None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES = {"llama8b_32k": 110.4e6}      # profiles/decode_bf16_llama8b_32k.md
+NCU_TRAFFIC_BYTES = {"llama8b_32k": 109.3e6, "llama8b_4x128k": 1391.7e6}      # profiles/decode_bf16_llama8b_32k.md
 
 
 def measured_peak():
