@@ -44,7 +44,7 @@ def popcounts(mask_i32: torch.Tensor) -> torch.Tensor:
     return cnt
 
 
-def check_unit(wl, cache, out, b, h, keep, lens):
+def check_unit(wl, cache, out, b, h, keep, lens, keep_v=0):
     """Full oracle parity of one (sequence, KV head) unit, including its G query heads' outputs."""
     Bn, Hq, Hkv, W, D, S = wl.shape
     G = Hq // Hkv
@@ -56,7 +56,8 @@ def check_unit(wl, cache, out, b, h, keep, lens):
     _, a = oracle.window_mean(q_win, 1)
     assert np.array_equal(cache.qnorm[b, h].cpu().numpy(), a[0, 0])
     c = oracle.compress(k, [n], keep, a)
-    ref, _ = oracle.decode_attn(q, k, v, [n], c["mask"], c["mu"], a)
+    c["vmask"] = oracle.prune_values(v, [n], keep_v) if 0 < keep_v < 128 else None
+    ref, _ = oracle.decode_attn(q, k, v, [n], c["mask"], c["mu"], a, vmask=c["vmask"])
     return c, ref[0]
 
 
@@ -157,3 +158,37 @@ def test_config5_qwen_paged_variable_lengths(ratio):
             assert d <= TOL, f"ratio {ratio} layer {layer} unit ({b},{h}) max|delta| {d:.3e}"
         del wl, cache, u
         torch.cuda.empty_cache()
+
+
+def test_config5_qwen_paged_with_value_pruning():
+    """Layer 0 of the Qwen-shaped configuration with (0.5 + 0.5) key + value channel pruning."""
+    keep = keep_v = inputs.keep_count(128, 0.5)
+    wl = inputs.config_workload(4, device="cuda", seed_offset=0)
+    Bn, Hq, Hkv, W, D, S = wl.shape
+    lens = wl.seq_lens.tolist()
+    order = np.argsort(lens)
+    sample = [int(order[0]), int(order[-1])]
+    for b in sample:
+        sub = inputs.Workload(q_win=wl.q_win[b:b + 1], k=wl.k[b:b + 1, :, :lens[b]], v=wl.v[b:b + 1],
+                              q=wl.q[b:b + 1], seq_lens=wl.seq_lens[b:b + 1], dtype=wl.dtype, meta={})
+        inputs.enforce_saliency_gap(sub, keep)
+    table, n_pages = permuted_block_table(Bn, Hkv, lens, "cuda", seed=4242)
+    cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
+                       max_tokens=S, block_table=table, n_pool_pages=n_pages, keep_v=keep_v)
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    out = cache.decode(wl.q)
+    assert cache.status() == 0
+    G = Hq // Hkv
+    u = cache.unpack(want_vals=False, want_v=False, want_vmask=True)
+    valid = torch.arange(S, device="cuda")[None, None, :] < wl.seq_lens[:, None, None]
+    for name, want in (("mask", keep), ("vmask", keep_v)):
+        pc = popcounts(u[name])
+        assert bool((pc[valid.expand_as(pc)] == want).all()) and bool((pc[~valid.expand_as(pc)] == 0).all())
+    for b in sample:
+        h = b % Hkv
+        c, ref = check_unit(wl, cache, out, b, h, keep, lens, keep_v=keep_v)
+        n = lens[b]
+        assert np.array_equal(u["mask"][b, h, :n].cpu().numpy().view(np.uint32), c["mask"][0, 0])
+        assert np.array_equal(u["vmask"][b, h, :n].cpu().numpy().view(np.uint32), c["vmask"][0, 0])
+        d = float(np.abs(out[b, h * G:(h + 1) * G].cpu().numpy() - ref).max())
+        assert d <= TOL, f"unit ({b},{h}) max|delta| {d:.3e}"

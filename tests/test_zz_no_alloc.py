@@ -25,16 +25,17 @@ def built():
     B.lib()
 
 
-@pytest.mark.parametrize("dtype,Bn,Hq,Hkv,lens,keep", [
-    ("bf16", 2, 16, 4, [2100, 333], 64),        # several CTAs share a unit: partials and tickets in use
-    ("bf16", 1, 28, 4, [5000], 38),
-    ("f32", 2, 4, 2, [700, 64], 25),
+@pytest.mark.parametrize("dtype,Bn,Hq,Hkv,lens,keep,keep_v", [
+    ("bf16", 2, 16, 4, [2100, 333], 64, 0),     # several CTAs share a unit: partials and tickets in use
+    ("bf16", 1, 28, 4, [5000], 38, 0),
+    ("f32", 2, 4, 2, [700, 64], 25, 0),
+    ("bf16", 2, 16, 4, [2100, 333], 64, 64),    # pruned value rows
 ])
-def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, keep):
+def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, keep, keep_v):
     wl = inputs.make_workload(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=lens, window=16, dtype=dtype,
                               sigma_s=1.0 if dtype == "bf16" else 0.5, seed=321, device="cuda")
     cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=16, keep=keep, dtype=dtype,
-                       max_tokens=max(lens))
+                       max_tokens=max(lens), keep_v=keep_v)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     lse_ref = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
     ref = cache.decode(wl.q, lse=lse_ref)
