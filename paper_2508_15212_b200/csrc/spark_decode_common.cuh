@@ -332,15 +332,15 @@ __device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctr
 {
     id0 = -1; id1 = -1;
     if (!active) return;
-    const int max_tokens = A.max_blocks * kPageTokens;
     const Segment s = locate(C.prefix, A.B, A.Hkv, g, c1);
-    const int len = clamp_len(A.lens[s.b], max_tokens);
-    const int nblk = (len + kPageTokens - 1) / kPageTokens;
     const int32_t* bt = A.block_table + (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
     id0 = bt[A.pps * s.i0];
-    if (A.pps == 2 && 2 * s.i0 + 1 < nblk) {
-        id1 = bt[2 * s.i0 + 1];
-        if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
+    if (A.pps == 2) {                                       // second page of the step, if the sequence has one
+        const int len = clamp_len(A.lens[s.b], A.max_blocks * kPageTokens);
+        if (2 * s.i0 + 1 < (len + kPageTokens - 1) / kPageTokens) {
+            id1 = bt[2 * s.i0 + 1];
+            if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
+        }
     }
     if (id0 < 0 || id0 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id0 = 0; }
 }
