@@ -12,8 +12,9 @@
 //   evict_scores_kernel<pass 1>  per 128-token tile and query row: max and sum of exp of the scores
 //   evict_rowstats_kernel        merge the tile partials into the row's softmax normaliser
 //   evict_scores_kernel<pass 2>  recompute the tile's scores, accumulate the column sums = votes
-//   evict_select_kernel          pooled max, exact top-k by radix select on the float bit pattern,
-//                                ordered compaction into kept_tokens
+//   evict_pool_kernel            pooled max of the votes, as order-preserving integer keys
+//   evict_hist_kernel<0..3>      radix select of the k-th largest key, one byte per pass, all SMs
+//   evict_count / compact        ordered compaction of the kept positions into kept_tokens
 // Column sums are accumulated inside one CTA in a fixed order, so the votes are reproducible.
 #include "spark_common.cuh"
 
@@ -35,6 +36,9 @@ struct EvictArgs {
     float* rowstat;      // [units][R][2]
     float* votes;        // [units][S_max]
     unsigned* pooled;    // [units][S_max] pooled votes as order-preserving keys
+    int* hist;           // [units][4][256] radix-select histograms, one per pass
+    int* counts;         // [units][n_chunks][2] keys above / equal to the threshold per 4096-token chunk
+    int n_chunks;
     int32_t* kept;       // [units][budget]
     int32_t* packed_lens;
     int* status;
@@ -188,6 +192,8 @@ __global__ void __launch_bounds__(256) evict_pool_kernel(EvictArgs A)
     const int S = min(A.seq_lens[b], A.S_max);
     if (S <= A.budget) return;
     const int P = S - A.W, half = (A.pool - 1) / 2;
+    if (blockIdx.x == 0)                                   // fresh histograms for this call's radix select
+        for (int i = threadIdx.x; i < 1024; i += blockDim.x) A.hist[static_cast<int64_t>(b * A.Hkv + h) * 1024 + i] = 0;
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= P) return;
     const int64_t base = static_cast<int64_t>(b * A.Hkv + h) * A.S_max;
@@ -197,108 +203,218 @@ __global__ void __launch_bounds__(256) evict_pool_kernel(EvictArgs A)
     A.pooled[base + t] = __float_as_uint(m);
 }
 
-// One CTA per unit: exact top-k of the pooled votes, ordered compaction.
-__global__ void __launch_bounds__(1024) evict_select_kernel(EvictArgs A)
+// ------------------------------------------------------------------------------------------------
+// Exact top-k of the pooled votes and ordered compaction, spread over the whole GPU.
+//
+// The k-th largest key of a unit is found by a radix select, 8 bits per pass: every CTA histograms its
+// 4096-token chunk into shared memory and adds the non-empty bins to the unit's histogram of that pass
+// (integer atomics: the result does not depend on arrival order).  The choice made by each finished pass
+// (the byte of the threshold, the rank left inside that bin) is recomputed from the stored histograms by
+// whoever needs it, so there is no separate "pick" launch.  After four passes the threshold key and the
+// number of equal keys to admit (lowest positions first) are known; a counting kernel gives every chunk
+// its base position and the compaction kernel writes the kept positions in order.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSelChunk = 4096;
+constexpr int kSelThreads = 256;
+constexpr int kSelPerThread = kSelChunk / kSelThreads;
+
+struct SelState { unsigned prefix, mask; int need; };
+
+// Replays the first `passes` picks from the unit's histograms ([4][256]).  One full warp.
+__device__ __forceinline__ SelState select_state(const int* hist, int passes, int k, int lane)
 {
-    __shared__ int hist[256];
-    __shared__ int scan[32];
-    __shared__ unsigned s_prefix, s_mask;
-    __shared__ int s_need, s_base_kept, s_base_eq;
-    const int h = blockIdx.x, b = blockIdx.y;
+    SelState s;
+    s.prefix = 0u; s.mask = 0u; s.need = k;
+    for (int p = 0; p < passes; ++p) {
+        const int* hp = hist + p * 256;
+        const int shift = 24 - 8 * p;
+        int loc[8], sum = 0;                              // lane l: bins 255 - 8l, 254 - 8l, ... (descending)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { loc[i] = hp[255 - 8 * lane - i]; sum += loc[i]; }
+        int inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += n; }
+        const unsigned cross = __ballot_sync(0xffffffffu, inc >= s.need);
+        const int src = cross ? __ffs(cross) - 1 : 31;   // lane whose bins contain the need-th largest key
+        int bin = 0, left = 0;
+        if (lane == src) {
+            int need = s.need - (inc - sum), i = 0;
+            for (; i < 7; ++i) { if (loc[i] >= need) break; need -= loc[i]; }
+            bin = 255 - 8 * lane - i;
+            left = need;
+        }
+        bin = __shfl_sync(0xffffffffu, bin, src);
+        left = __shfl_sync(0xffffffffu, left, src);
+        s.need = left;                                    // rank inside the chosen bin
+        s.prefix |= static_cast<unsigned>(bin) << shift;
+        s.mask |= 255u << shift;
+    }
+    return s;
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(kSelThreads) evict_hist_kernel(EvictArgs A)
+{
+    __shared__ int sh[256];
+    __shared__ SelState st;
+    const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int S = min(A.seq_lens[b], A.S_max);
+    if (S <= A.budget) return;
+    const int P = S - A.W, k = A.budget - A.W, t0 = chunk * kSelChunk;
+    if (t0 >= P) return;
+    const int unit = b * A.Hkv + h, tid = threadIdx.x, lane = tid & 31;
+    int* hist = A.hist + static_cast<int64_t>(unit) * 1024;
+    sh[tid] = 0;
+    if (tid < 32) {
+        const SelState s = select_state(hist, PASS, k, lane);
+        if (lane == 0) st = s;
+    }
+    __syncthreads();
+    const unsigned prefix = st.prefix, mask = st.mask;
+    constexpr int shift = 24 - 8 * PASS;
+    const unsigned* pooled = A.pooled + static_cast<int64_t>(unit) * A.S_max;
+#pragma unroll 4
+    for (int i = 0; i < kSelPerThread; ++i) {              // whole warps iterate together (votes below)
+        const int t = t0 + i * kSelThreads + tid;
+        const unsigned key = t < P ? pooled[t] : 0u;
+        const bool in = t < P && (key & mask) == prefix;
+        const unsigned bin = (key >> shift) & 255u;
+        // lanes that hit the same bin add once: keys of neighbouring tokens mostly share their top bytes
+        const unsigned active = __ballot_sync(0xffffffffu, in);
+        if (in) {
+            const unsigned peers = __match_any_sync(active, bin);
+            if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], __popc(peers));
+        }
+    }
+    __syncthreads();
+    if (sh[tid]) atomicAdd(&hist[PASS * 256 + tid], sh[tid]);
+}
+
+// counts[unit][chunk] = (keys above the threshold, keys equal to it) in the chunk
+__global__ void __launch_bounds__(kSelThreads) evict_count_kernel(EvictArgs A)
+{
+    __shared__ SelState st;
+    __shared__ int red[2][kSelThreads / 32];
+    const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int S = min(A.seq_lens[b], A.S_max);
+    if (S <= A.budget) return;
+    const int P = S - A.W, k = A.budget - A.W, t0 = chunk * kSelChunk;
+    if (t0 >= P) return;
+    const int unit = b * A.Hkv + h, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid < 32) {
+        const SelState s = select_state(A.hist + static_cast<int64_t>(unit) * 1024, 4, k, lane);
+        if (lane == 0) st = s;
+    }
+    __syncthreads();
+    const unsigned thr = st.prefix;
+    const unsigned* pooled = A.pooled + static_cast<int64_t>(unit) * A.S_max;
+    int gt = 0, eq = 0;
+#pragma unroll 4
+    for (int i = 0; i < kSelPerThread; ++i) {
+        const int t = t0 + i * kSelThreads + tid;
+        if (t < P) { const unsigned key = pooled[t]; gt += key > thr; eq += key == thr; }
+    }
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    eq = __reduce_add_sync(0xffffffffu, eq);
+    if (lane == 0) { red[0][warp] = gt; red[1][warp] = eq; }
+    __syncthreads();
+    if (tid == 0) {
+        int g = 0, e = 0;
+        for (int w = 0; w < kSelThreads / 32; ++w) { g += red[0][w]; e += red[1][w]; }
+        int* c = A.counts + (static_cast<int64_t>(unit) * A.n_chunks + chunk) * 2;
+        c[0] = g; c[1] = e;
+    }
+}
+
+// Ordered compaction: thread i of the chunk's CTA owns 16 consecutive tokens.  Also publishes packed_lens
+// and handles sequences that are kept whole.
+__global__ void __launch_bounds__(kSelThreads) evict_compact_kernel(EvictArgs A)
+{
+    __shared__ SelState st;
+    __shared__ int s_base_kept, s_base_eq;
+    __shared__ int scan_eq[kSelThreads / 32], scan_keep[kSelThreads / 32];
+    const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int S = A.seq_lens[b];
     if (S < 0 || S > A.S_max) {
-        if (threadIdx.x == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        if (chunk == 0 && tid == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
         S = S < 0 ? 0 : A.S_max;
     }
     const int unit = b * A.Hkv + h;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t* kept = A.kept + static_cast<int64_t>(unit) * A.budget;
-    if (h == 0 && tid == 0) A.packed_lens[b] = S < A.budget ? (S < 0 ? 0 : S) : A.budget;
-    if (S <= A.budget) {
-        for (int t = tid; t < A.budget; t += blockDim.x) kept[t] = t < S ? t : -1;
+    if (chunk == 0 && h == 0 && tid == 0) A.packed_lens[b] = S < A.budget ? S : A.budget;
+    if (S <= A.budget) {                                  // kept whole
+        for (int t = chunk * kSelChunk + tid; t < min(A.budget, (chunk + 1) * kSelChunk); t += kSelThreads)
+            kept[t] = t < S ? t : -1;
+        if (chunk == 0)                                   // budget beyond the chunked range (short max_seq_tokens)
+            for (int t = A.n_chunks * kSelChunk + tid; t < A.budget; t += kSelThreads) kept[t] = t < S ? t : -1;
         return;
     }
-    const int P = S - A.W, k = A.budget - A.W;
+    const int P = S - A.W, k = A.budget - A.W, t0 = chunk * kSelChunk;
+    if (chunk == 0)
+        for (int w = tid; w < A.W; w += kSelThreads) kept[k + w] = P + w;
+    if (t0 >= P) return;
+    if (tid < 32) {
+        const SelState s = select_state(A.hist + static_cast<int64_t>(unit) * 1024, 4, k, lane);
+        if (lane == 0) {
+            st = s;
+            // position of this chunk's first kept token and number of equal keys before the chunk
+            const int* c = A.counts + static_cast<int64_t>(unit) * A.n_chunks * 2;
+            int base_kept = 0, base_eq = 0;
+            for (int cc = 0; cc < chunk; ++cc) {
+                const int take = min(c[2 * cc + 1], max(0, s.need - base_eq));
+                base_kept += c[2 * cc] + take;
+                base_eq += c[2 * cc + 1];
+            }
+            s_base_kept = base_kept; s_base_eq = base_eq;
+        }
+    }
+    __syncthreads();
+    const unsigned thr = st.prefix;
+    const int need_eq = st.need;
     const unsigned* pooled = A.pooled + static_cast<int64_t>(unit) * A.S_max;
-    auto pooled_key = [&](int t) -> unsigned { return pooled[t]; };
-    // radix select of the k-th largest key, 8 bits per pass
-    if (tid == 0) { s_prefix = 0; s_mask = 0; s_need = k; }
-    __syncthreads();
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0;
-        __syncthreads();
-        const unsigned prefix = s_prefix, mask = s_mask;
-        for (int t0 = 0; t0 < P; t0 += blockDim.x) {        // all lanes iterate together (warp votes below)
-            const int t = t0 + tid;
-            const unsigned key = t < P ? pooled_key(t) : 0u;
-            const bool in = t < P && (key & mask) == prefix;
-            const unsigned bin = (key >> shift) & 255u;
-            // lanes that hit the same bin add once: keys of neighbouring tokens mostly share their top bytes
-            const unsigned active = __ballot_sync(0xffffffffu, in);
-            if (in) {
-                const unsigned peers = __match_any_sync(active, bin);
-                if (lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
-            }
-        }
-        __syncthreads();
-        if (tid == 0) {
-            int need = s_need, bin = 255;
-            for (; bin > 0; --bin) {
-                if (hist[bin] >= need) break;
-                need -= hist[bin];
-            }
-            s_need = need;                                  // rank inside the chosen bin
-            s_prefix = prefix | (static_cast<unsigned>(bin) << shift);
-            s_mask = mask | (255u << shift);
-        }
-        __syncthreads();
+    const int tb = t0 + tid * kSelPerThread;
+    unsigned key[kSelPerThread];
+    int eq_cnt = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i) {
+        key[i] = (tb + i < P) ? pooled[tb + i] : 0u;
+        eq_cnt += (tb + i < P && key[i] == thr) ? 1 : 0;
     }
-    const unsigned thr = s_prefix;                          // k-th largest key; s_need of the keys equal to it are kept
-    const int need_eq = s_need;
-    if (tid == 0) { s_base_kept = 0; s_base_eq = 0; }
+    // exclusive scan of eq_cnt over the CTA's threads (threads are in position order)
+    int v = eq_cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += n; }
+    if (lane == 31) scan_eq[warp] = v;
     __syncthreads();
-    for (int c0 = 0; c0 < P; c0 += blockDim.x) {
-        const int t = c0 + tid;
-        const unsigned key = t < P ? pooled_key(t) : 0u;
-        const int eq = (t < P && key == thr) ? 1 : 0;
-        // exclusive scan of eq over the block
-        int v = eq;
+    int eq_rank = s_base_eq + v - eq_cnt;
+    for (int w = 0; w < warp; ++w) eq_rank += scan_eq[w];
+    unsigned keep_bits = 0u;
+    int keep_cnt = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += n; }
-        if (lane == 31) scan[warp] = v;
-        __syncthreads();
-        if (warp == 0) {
-            int s = scan[lane];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += n; }
-            scan[lane] = s;
-        }
-        __syncthreads();
-        const int eq_rank = s_base_eq + (warp ? scan[warp - 1] : 0) + v - eq;
-        const int eq_total = scan[31];
-        const int keep = (t < P && (key > thr || (eq && eq_rank < need_eq))) ? 1 : 0;
-        __syncthreads();
-        int u = keep;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, u, o); if (lane >= o) u += n; }
-        if (lane == 31) scan[warp] = u;
-        __syncthreads();
-        if (warp == 0) {
-            int s = scan[lane];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, s, o); if (lane >= o) s += n; }
-            scan[lane] = s;
-        }
-        __syncthreads();
-        const int pos = s_base_kept + (warp ? scan[warp - 1] : 0) + u - keep;
-        if (keep && pos < k) kept[pos] = t;
-        const int kept_total = scan[31];
-        __syncthreads();
-        if (tid == 0) { s_base_kept += kept_total; s_base_eq += eq_total; }
-        __syncthreads();
+    for (int i = 0; i < kSelPerThread; ++i) {
+        const bool live = tb + i < P;
+        const bool eq = live && key[i] == thr;
+        const bool keep = live && (key[i] > thr || (eq && eq_rank < need_eq));
+        eq_rank += eq ? 1 : 0;
+        keep_bits |= keep ? (1u << i) : 0u;
+        keep_cnt += keep ? 1 : 0;
     }
-    for (int w = tid; w < A.W; w += blockDim.x) kept[k + w] = P + w;
-    if (tid == 0 && s_base_kept != k) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+    int u = keep_cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int n = __shfl_up_sync(0xffffffffu, u, o); if (lane >= o) u += n; }
+    if (lane == 31) scan_keep[warp] = u;
+    __syncthreads();
+    int pos = s_base_kept + u - keep_cnt;
+    for (int w = 0; w < warp; ++w) pos += scan_keep[w];
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if ((keep_bits >> i) & 1u) {
+            if (pos < k) kept[pos] = tb + i;
+            ++pos;
+        }
+    // the thread that owns the last prefix token sees the total
+    if (tb <= P - 1 && P - 1 < tb + kSelPerThread && pos != k) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
 }
 
 bool evict_tc_supported(const spark_params& p);
@@ -315,6 +431,8 @@ size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens)
     size_t bytes = units * R * tiles * 2 * sizeof(float);
     bytes += units * R * 2 * sizeof(float);
     bytes += 2 * units * static_cast<size_t>(max_seq_tokens) * sizeof(float);      // votes, pooled keys
+    const size_t chunks = (max_seq_tokens + kSelChunk - 1) / kSelChunk;
+    bytes += units * (1024 + 2 * (chunks ? chunks : 1)) * sizeof(int);             // select histograms, chunk counts
     return (bytes + 255) / 256 * 256;
 }
 
@@ -334,6 +452,10 @@ spark_status launch_evict(const spark_params& p, const void* q_win, const void* 
     A.rowstat = A.partial + units * R * A.n_tiles * 2;
     A.votes = A.rowstat + units * R * 2;
     A.pooled = reinterpret_cast<unsigned*>(A.votes + units * static_cast<size_t>(max_seq_tokens));
+    A.hist = reinterpret_cast<int*>(A.pooled + units * static_cast<size_t>(max_seq_tokens));
+    A.counts = A.hist + units * 1024;
+    A.n_chunks = (max_seq_tokens + kSelChunk - 1) / kSelChunk;
+    if (A.n_chunks < 1) A.n_chunks = 1;
     A.kept = kept_tokens; A.packed_lens = packed_lens;
     const size_t smem = (static_cast<size_t>(kEvTile + kEvRows) * kEvStride + kEvTile) * sizeof(float);
     const dim3 grid(A.n_tiles, p.n_kv_heads, p.batch), ugrid(p.n_kv_heads, p.batch);
@@ -355,11 +477,17 @@ spark_status launch_evict(const spark_params& p, const void* q_win, const void* 
         else evict_scores_kernel<float, 2><<<grid, kEvThreads, smem, stream>>>(A);
         *launches += 3;
     }
+    const dim3 sgrid(A.n_chunks, p.n_kv_heads, p.batch);
     if (max_seq_tokens > p.token_budget) {
         evict_pool_kernel<<<dim3((max_seq_tokens + 255) / 256, p.n_kv_heads, p.batch), 256, 0, stream>>>(A);
-        ++*launches;
+        evict_hist_kernel<0><<<sgrid, kSelThreads, 0, stream>>>(A);
+        evict_hist_kernel<1><<<sgrid, kSelThreads, 0, stream>>>(A);
+        evict_hist_kernel<2><<<sgrid, kSelThreads, 0, stream>>>(A);
+        evict_hist_kernel<3><<<sgrid, kSelThreads, 0, stream>>>(A);
+        evict_count_kernel<<<sgrid, kSelThreads, 0, stream>>>(A);
+        *launches += 6;
     }
-    evict_select_kernel<<<ugrid, 1024, 0, stream>>>(A);
+    evict_compact_kernel<<<sgrid, kSelThreads, 0, stream>>>(A);
     ++*launches;
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
