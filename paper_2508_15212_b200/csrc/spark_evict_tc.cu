@@ -87,6 +87,22 @@ __device__ __forceinline__ void tc_ld32(unsigned taddr, float (&v)[32])
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 128 consecutive columns of this thread's tensor-memory lane: two 64-column loads and one wait in a single
+// statement, so nothing reads the registers before the wait.
+__device__ __forceinline__ void tc_ld128(unsigned taddr, float (&v)[128])
+{
+    unsigned r[128];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%128];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%64,%65,%66,%67,%68,%69,%70,%71,%72,%73,%74,%75,%76,%77,%78,%79,%80,%81,%82,%83,%84,%85,%86,%87,%88,%89,%90,%91,%92,%93,%94,%95,%96,%97,%98,%99,%100,%101,%102,%103,%104,%105,%106,%107,%108,%109,%110,%111,%112,%113,%114,%115,%116,%117,%118,%119,%120,%121,%122,%123,%124,%125,%126,%127}, [%129];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95]), "=r"(r[96]), "=r"(r[97]), "=r"(r[98]), "=r"(r[99]), "=r"(r[100]), "=r"(r[101]), "=r"(r[102]), "=r"(r[103]), "=r"(r[104]), "=r"(r[105]), "=r"(r[106]), "=r"(r[107]), "=r"(r[108]), "=r"(r[109]), "=r"(r[110]), "=r"(r[111]), "=r"(r[112]), "=r"(r[113]), "=r"(r[114]), "=r"(r[115]), "=r"(r[116]), "=r"(r[117]), "=r"(r[118]), "=r"(r[119]), "=r"(r[120]), "=r"(r[121]), "=r"(r[122]), "=r"(r[123]), "=r"(r[124]), "=r"(r[125]), "=r"(r[126]), "=r"(r[127])
+        : "r"(taddr), "r"(taddr + 64u)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 128; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // Copy `rows` rows of 128 bf16 channels (row i at src + i*stride elements; rows >= valid are zero) into
 // the two 64-channel swizzled blocks at dst (block 0 at dst, block 1 at dst + rows_alloc*128 bytes).
 __device__ __forceinline__ void tc_stage_rows(unsigned char* dst, int rows_alloc, const unsigned short* src, int64_t stride,
@@ -99,6 +115,23 @@ __device__ __forceinline__ void tc_stage_rows(unsigned char* dst, int rows_alloc
         const int kb = ch16 >> 3, c8 = ch16 & 7;
         *reinterpret_cast<uint4*>(dst + static_cast<size_t>(kb) * rows_alloc * 128 + r * 128 + ((c8 ^ (r & 7)) << 4)) = v;
     }
+}
+
+// The same copy for a key tile with 16-byte asynchronous copies (rows >= valid are zero-filled): the
+// caller commits the group and waits for it one tile later, so the load of tile i+1 runs under the MMAs
+// and the epilogue of tile i.
+__device__ __forceinline__ void tc_stage_rows_async(unsigned dst_u, int rows_alloc, const unsigned short* src, int64_t stride,
+                                                    int valid, int tid)
+{
+    for (int i = tid; i < rows_alloc * 16; i += kTcThreads) {
+        const int r = i >> 4, ch16 = i & 15;
+        const int kb = ch16 >> 3, c8 = ch16 & 7;
+        const bool live = r < valid;
+        const unsigned short* g = src + static_cast<int64_t>(live ? r : 0) * stride + ch16 * 8;
+        const unsigned d = dst_u + static_cast<unsigned>(kb) * rows_alloc * 128u + r * 128u + ((c8 ^ (r & 7)) << 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(g), "r"(live ? 16 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
 template <int PASS>
@@ -125,7 +158,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
 
     // operand tiles start on a 1024-byte boundary (the swizzle atom); the launch reserves the slack
     unsigned char* q_s = tc_smem + ((1024u - (tc_smem_u32(tc_smem) & 1023u)) & 1023u);   // [2][Rpad][128 B]
-    unsigned char* k_s = q_s + static_cast<size_t>(Rpad) * 256;                            // [2][128][128 B]
+    unsigned char* k_s = q_s + static_cast<size_t>(Rpad) * 256;                            // 2 buffers of [2][128][128 B]
     const int n_cols = (PASS == 1) ? Rpad : (Rn <= 128 ? 128 : 256);   // tensor-memory columns (power of two >= 32)
 
     if (warp == 0) {
@@ -149,7 +182,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const unsigned tmem = tmem_base_s;
-    const unsigned q_u = tc_smem_u32(q_s), k_u = tc_smem_u32(k_s);
+    const unsigned q_u = tc_smem_u32(q_s), k_u0 = tc_smem_u32(k_s);
+    const unsigned short* k_unit = static_cast<const unsigned short*>(A.k) + static_cast<int64_t>(b) * A.sb +
+                                   static_cast<int64_t>(h) * A.sh;
+    if (tile0 < tile1)                                     // first key tile in flight
+        tc_stage_rows_async(k_u0, kTcTile, k_unit + static_cast<int64_t>(tile0) * kTcTile * A.st, A.st,
+                            min(kTcTile, S - tile0 * kTcTile), tid);
 
     float run_m[2] = {-INFINITY, -INFINITY}, run_l[2] = {0.f, 0.f};       // pass 1: rows tid and 128 + tid
     unsigned phase = 0;
@@ -157,13 +195,15 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
 
     for (int tile = tile0; tile < tile1; ++tile) {
         const int t0 = tile * kTcTile;
-        const int valid = min(kTcTile, S - t0);
-        tc_stage_rows(k_s, kTcTile, static_cast<const unsigned short*>(A.k) + static_cast<int64_t>(b) * A.sb +
-                                        static_cast<int64_t>(h) * A.sh + static_cast<int64_t>(t0) * A.st,
-                      A.st, valid, tid);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy stores -> tensor-core reads
+        const unsigned k_u = k_u0 + static_cast<unsigned>((tile - tile0) & 1) * (kTcTile * 256u);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");             // this tile's keys have landed
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> tensor-core reads
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
+        if (tile + 1 < tile1)                                            // next tile into the other buffer
+            tc_stage_rows_async(k_u0 + static_cast<unsigned>((tile + 1 - tile0) & 1) * (kTcTile * 256u), kTcTile,
+                                k_unit + static_cast<int64_t>(t0 + kTcTile) * A.st, A.st,
+                                min(kTcTile, S - (t0 + kTcTile)), tid);
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (PASS == 1) {
@@ -202,25 +242,22 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
                     const bool row_ok = row < R;
                     const int last = P + (row_ok ? row % A.W : 0);
                     float m = run_m[mb], l = run_l[mb];
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kTcTile; c0 += 32) {
-                        float v[32];
-                        tc_ld32(lane_addr + mb * 128 + c0, v);
-                        float cm = -INFINITY;
+                    float v[kTcTile];
+                    tc_ld128(lane_addr + mb * 128, v);
+                    float cm = -INFINITY;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int t = t0 + c0 + i;
-                            v[i] = (row_ok && t <= last && t < S) ? v[i] * scale : -INFINITY;
-                            cm = fmaxf(cm, v[i]);
-                        }
-                        if (cm > -INFINITY) {
-                            const float mn = fmaxf(m, cm);
-                            float add = 0.f;
+                    for (int i = 0; i < kTcTile; ++i) {
+                        const int t = t0 + i;
+                        v[i] = (row_ok && t <= last && t < S) ? v[i] * scale : -INFINITY;
+                        cm = fmaxf(cm, v[i]);
+                    }
+                    if (cm > -INFINITY) {
+                        const float mn = fmaxf(m, cm);
+                        float add[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) add += tc_ex2(v[i] - mn);          // 2^(-inf) = 0 for masked keys
-                            l = l * tc_ex2(m - mn) + add;
-                            m = mn;
-                        }
+                        for (int i = 0; i < kTcTile; ++i) add[i & 3] += tc_ex2(v[i] - mn);    // 2^(-inf) = 0 for masked keys
+                        l = l * tc_ex2(m - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
+                        m = mn;
                     }
                     run_m[mb] = m; run_l[mb] = l;
                 }
@@ -228,11 +265,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
                 const int t = t0 + tid;
                 float vote = 0.f;
 #pragma unroll 1
-                for (int c0 = 0; c0 < Rn; c0 += 32) {
-                    float v[32];
-                    tc_ld32(lane_addr + c0, v);
+                for (int c0 = 0; c0 < Rn; c0 += 128) {
+                    float v[128];
+                    tc_ld128(lane_addr + c0, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < 128; ++i) {
                         const int row = c0 + i;
                         if (row < R) vote += tc_ex2(fmaf(v[i], scale, -row_m[row])) * row_il[row];
                     }
@@ -297,10 +334,20 @@ spark_status launch_evict_votes_tc(const spark_params& p, const void* q_win, con
     A.q_win = q_win; A.k = k; A.sb = sb; A.sh = sh; A.st = st; A.seq_lens = seq_lens;
     A.Hq = p.n_q_heads; A.Hkv = p.n_kv_heads; A.W = p.window; A.budget = p.token_budget; A.S_max = max_seq_tokens;
     const int n_tiles = (max_seq_tokens + kTcTile - 1) / kTcTile;
-    A.tiles_per_cta = 8;
+    // Two CTAs are resident per SM; a CTA pays a fixed start-up (tensor-memory allocation, the query
+    // block, the first key tile), so the tiles are cut into about one wave of CTAs, at least 8 tiles each.
+    int dev = 0, n_sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    const int64_t units = static_cast<int64_t>(p.batch) * p.n_kv_heads;
+    const int64_t wave = 2 * static_cast<int64_t>(n_sms);
+    int64_t per = (static_cast<int64_t>(n_tiles) * units + wave - 1) / wave;
+    if (per < 8) per = 8;
+    if (per > n_tiles) per = n_tiles > 0 ? n_tiles : 1;
+    A.tiles_per_cta = static_cast<int>(per);
     A.parts = (n_tiles + A.tiles_per_cta - 1) / A.tiles_per_cta;
     A.partial = partial; A.rowstat = rowstat; A.votes = votes; A.status = status;
-    const size_t smem = static_cast<size_t>(Rpad) * 256 + kTcTile * 256 + 1024;
+    const size_t smem = static_cast<size_t>(Rpad) * 256 + 2 * kTcTile * 256 + 1024;     // queries, two key buffers, alignment slack
     if (cudaFuncSetAttribute(evict_scores_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
         cudaFuncSetAttribute(evict_scores_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
         return SPARK_ERR_CUDA;
