@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
     extern __shared__ __align__(1024) unsigned char tc_smem[];
     __shared__ __align__(8) uint64_t mma_bar;
     __shared__ unsigned tmem_base_s;
-    __shared__ float row_m[256], row_il[256];
+    __shared__ __align__(16) float row_c[256];              // pass 2: log2-domain softmax offset of each query row
 
     const int part = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int S = min(A.seq_lens[b], A.S_max);
@@ -172,12 +172,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
     // query rows of the group: row = g*W + w  ->  q_win[b][h*G+g][w][:]  (contiguous over (g, w))
     tc_stage_rows(q_s, Rpad, static_cast<const unsigned short*>(A.q_win) + (static_cast<int64_t>(b) * A.Hq + h * G) * A.W * kHeadDim,
                   kHeadDim, R, tid);
-    if (PASS == 2)
-        for (int r = tid; r < 256; r += kTcThreads) {
-            const bool ok = r < R;
-            row_m[r] = ok ? A.rowstat[(static_cast<int64_t>(unit) * R + r) * 2] : 0.f;
-            row_il[r] = ok ? 1.0f / A.rowstat[(static_cast<int64_t>(unit) * R + r) * 2 + 1] : 0.f;
-        }
+    if (PASS == 2)                                         // p = 2^(s - c), c = row max + log2(row sum); padding rows give 0
+        for (int r = tid; r < 256; r += kTcThreads)
+            row_c[r] = (r < R) ? A.rowstat[(static_cast<int64_t>(unit) * R + r) * 2] +
+                                     log2f(A.rowstat[(static_cast<int64_t>(unit) * R + r) * 2 + 1])
+                               : INFINITY;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -244,20 +243,34 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
                     float m = run_m[mb], l = run_l[mb];
                     float v[kTcTile];
                     tc_ld128(lane_addr + mb * 128, v);
-                    float cm = -INFINITY;
+                    if (t0 + kTcTile <= P + 1) {               // every key of the tile is visible to every window row
+                        if (row_ok) {
+                            float c4[4] = {v[0], v[1], v[2], v[3]};
 #pragma unroll
-                    for (int i = 0; i < kTcTile; ++i) {
-                        const int t = t0 + i;
-                        v[i] = (row_ok && t <= last && t < S) ? v[i] * scale : -INFINITY;
-                        cm = fmaxf(cm, v[i]);
-                    }
-                    if (cm > -INFINITY) {
-                        const float mn = fmaxf(m, cm);
-                        float add[4] = {0.f, 0.f, 0.f, 0.f};
+                            for (int i = 4; i < kTcTile; ++i) c4[i & 3] = fmaxf(c4[i & 3], v[i]);
+                            const float mn = fmaxf(m, fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3])) * scale);
+                            float add[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int i = 0; i < kTcTile; ++i) add[i & 3] += tc_ex2(v[i] - mn);    // 2^(-inf) = 0 for masked keys
-                        l = l * tc_ex2(m - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
-                        m = mn;
+                            for (int i = 0; i < kTcTile; ++i) add[i & 3] += tc_ex2(fmaf(v[i], scale, -mn));
+                            l = l * tc_ex2(m - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
+                            m = mn;
+                        }
+                    } else {
+                        float cm = -INFINITY;
+#pragma unroll
+                        for (int i = 0; i < kTcTile; ++i) {
+                            const int t = t0 + i;
+                            v[i] = (row_ok && t <= last && t < S) ? v[i] * scale : -INFINITY;
+                            cm = fmaxf(cm, v[i]);
+                        }
+                        if (cm > -INFINITY) {
+                            const float mn = fmaxf(m, cm);
+                            float add[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                            for (int i = 0; i < kTcTile; ++i) add[i & 3] += tc_ex2(v[i] - mn);    // 2^(-inf) = 0 for masked keys
+                            l = l * tc_ex2(m - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
+                            m = mn;
+                        }
                     }
                     run_m[mb] = m; run_l[mb] = l;
                 }
@@ -268,11 +281,16 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
                 for (int c0 = 0; c0 < Rn; c0 += 128) {
                     float v[128];
                     tc_ld128(lane_addr + c0, v);
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) {
-                        const int row = c0 + i;
-                        if (row < R) vote += tc_ex2(fmaf(v[i], scale, -row_m[row])) * row_il[row];
+                    for (int i = 0; i < 128; i += 4) {
+                        const float4 c = *reinterpret_cast<const float4*>(row_c + c0 + i);     // same address for all threads
+                        acc[0] += tc_ex2(fmaf(v[i], scale, -c.x));
+                        acc[1] += tc_ex2(fmaf(v[i + 1], scale, -c.y));
+                        acc[2] += tc_ex2(fmaf(v[i + 2], scale, -c.z));
+                        acc[3] += tc_ex2(fmaf(v[i + 3], scale, -c.w));
                     }
+                    vote += (acc[0] + acc[1]) + (acc[2] + acc[3]);
                 }
                 if (t < S) A.votes[static_cast<int64_t>(unit) * A.S_max + t] = (t < P) ? vote : 0.f;
             }
