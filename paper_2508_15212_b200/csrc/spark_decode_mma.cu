@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
             if (ok) {
                 // ---------------- scores of the page's 16 tokens (rows r and r+8) ----------------
                 float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f}, d3[4] = {0.f, 0.f, 0.f, 0.f};
-                unsigned vaddr[2], w[2];
+                unsigned vaddr[2], vaddr_hi[2], w[2];
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     const int tok = 8 * j + r;
@@ -327,6 +327,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                     t = __shfl_up_sync(kFull, x, 2, 4);
                     if (c >= 2) x += t;
                     vaddr[j] = page + (r * 2 + j) * 2 + (x - cnt) * 32;      // see val_offset: token r + 8j
+                    vaddr_hi[j] = vaddr[j] + __popc(w[j] & 0xffffu) * 32;    // upper half of the word walks on its own
                 }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -334,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
 #pragma unroll
                     for (int j = 0; j < 2; ++j)
                         expand_nibble(w[j], 1u << (4 * ks), 2u << (4 * ks), 4u << (4 * ks), 8u << (4 * ks),
-                                      vaddr[j], k0[j], k1[j], m0[j], m1[j]);
+                                      ks < 4 ? vaddr[j] : vaddr_hi[j], k0[j], k1[j], m0[j], m1[j]);
                     mma_bf16(d1, k0[0], k0[1], k1[0], k1[1], Bq[2 * ks], Bq[2 * ks + 1]);
                     mma_bf16(d2, m0[0], m0[1], m1[0], m1[1], Bp[2 * ks], Bp[2 * ks + 1]);
                     if (!kShared8) mma_bf16(d3, m0[0], m0[1], m1[0], m1[1], Bpl[2 * ks], Bpl[2 * ks + 1]);
