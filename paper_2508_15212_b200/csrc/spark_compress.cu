@@ -64,12 +64,14 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 //
 // The same routine prunes a value row (a = 1, so the key is |V[t][j]| itself): `vals_off` / `mask_off`
 // select the section that receives the kept entries and the mask, and mu is written only when
-// `mu_off` >= 0.
+// `mu_off` >= 0 (`inv_pruned` = 1 / (D - T), or 0 when nothing is pruned: the mean is taken as a product
+// in double, which rounds to the same float as the quotient except on a rounding boundary of the double).
 // ------------------------------------------------------------------------------------------------
 template <bool kBf16>
 __device__ __forceinline__ void pack_token(unsigned char* image, int esize, int vals_off, int mask_off, int mu_off,
                                            int p, int T, int lane,
-                                           const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4])
+                                           const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4],
+                                           double inv_pruned = 0.0)
 {
     const unsigned lt = (1u << lane) - 1u;
     float w[4];
@@ -149,8 +151,7 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int esize, int 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
     if (lane == 0)
-        reinterpret_cast<float*>(image + mu_off)[p] =
-            (T < kHeadDim) ? static_cast<float>(pruned / static_cast<double>(kHeadDim - T)) : 0.f;
+        reinterpret_cast<float*>(image + mu_off)[p] = static_cast<float>(pruned * inv_pruned);
 }
 
 // Key entries and value entries of one token into the page image (a lane owns channels 4*lane .. 4*lane+3;
@@ -175,7 +176,8 @@ __device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLa
         *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) =
             make_uint4(vraw[0], vraw[1], vraw[2], vraw[3]);
     }
-    pack_token<kBf16>(image, L.esize, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw);
+    const double inv_pruned = L.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - L.keep) : 0.0;   // folded by the compiler into one constant load per kernel
+    pack_token<kBf16>(image, L.esize, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned);
 }
 
 // A lane's four key and value entries of one token row (bit patterns).
