@@ -68,7 +68,7 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 // in double, which rounds to the same float as the quotient except on a rounding boundary of the double).
 // ------------------------------------------------------------------------------------------------
 template <bool kBf16>
-__device__ __forceinline__ void pack_token(unsigned char* image, int esize, int vals_off, int mask_off, int mu_off,
+__device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, int mask_off, int mu_off,
                                            int p, int T, int lane,
                                            const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4],
                                            double inv_pruned = 0.0)
@@ -133,7 +133,7 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int esize, int 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         if (kept[i]) {
-            unsigned char* dst = image + vals_off + val_offset(esize, p, slot);
+            unsigned char* dst = image + vals_off + val_offset(kBf16 ? 2 : 4, p, slot);
             if (kBf16) *reinterpret_cast<unsigned short*>(dst) = static_cast<unsigned short>(raw[i]);
             else *reinterpret_cast<unsigned*>(dst) = raw[i];
             ++slot;
@@ -154,47 +154,44 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int esize, int 
         reinterpret_cast<float*>(image + mu_off)[p] = static_cast<float>(pruned * inv_pruned);
 }
 
-// Key entries and value entries of one token into the page image (a lane owns channels 4*lane .. 4*lane+3;
-// `kraw` / `vraw` are the stored bit patterns of its key and value entries).
+// Key entries and value entries of one token row into the page image.  A lane owns channels 4*lane ..
+// 4*lane+3; `row` is the element offset of its first channel in k and v.  `inv_pruned` = 1 / (D - T)
+// (0 when T = D), computed once on the host.
 template <bool kBf16>
 __device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLayout& L, int p, int lane,
-                                              const float (&a)[4], const unsigned (&kraw)[4], const unsigned (&vraw)[4])
+                                              const float (&a)[4], const void* k, const void* v, int64_t row,
+                                              double inv_pruned)
 {
-    float kf[4], vf[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        kf[i] = __uint_as_float(kBf16 ? kraw[i] << 16 : kraw[i]);
-        vf[i] = __uint_as_float(kBf16 ? vraw[i] << 16 : vraw[i]);
-    }
-    if (L.keep_v < kHeadDim) {
-        const float one[4] = {1.f, 1.f, 1.f, 1.f};
-        pack_token<kBf16>(image, L.esize, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
-    } else if (kBf16) {
-        *reinterpret_cast<uint2*>(image + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) =
-            make_uint2(vraw[0] | (vraw[1] << 16), vraw[2] | (vraw[3] << 16));
-    } else {
-        *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) =
-            make_uint4(vraw[0], vraw[1], vraw[2], vraw[3]);
-    }
-    const double inv_pruned = L.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - L.keep) : 0.0;   // folded by the compiler into one constant load per kernel
-    pack_token<kBf16>(image, L.esize, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned);
-}
-
-// A lane's four key and value entries of one token row (bit patterns).
-template <bool kBf16>
-__device__ __forceinline__ void load_kv_row(const void* k, const void* v, int64_t row, unsigned (&kraw)[4], unsigned (&vraw)[4])
-{
+    unsigned kraw[4], vraw[4];
+    float kf[4];
     if (kBf16) {
         const uint2 kk = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(k) + row);
         const uint2 vv = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(v) + row);
         kraw[0] = kk.x & 0xffffu; kraw[1] = kk.x >> 16; kraw[2] = kk.y & 0xffffu; kraw[3] = kk.y >> 16;
-        vraw[0] = vv.x & 0xffffu; vraw[1] = vv.x >> 16; vraw[2] = vv.y & 0xffffu; vraw[3] = vv.y >> 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(kraw[i] << 16);
+        if (L.keep_v < kHeadDim) {
+            vraw[0] = vv.x & 0xffffu; vraw[1] = vv.x >> 16; vraw[2] = vv.y & 0xffffu; vraw[3] = vv.y >> 16;
+        } else {
+            *reinterpret_cast<uint2*>(image + L.v_off + v_chunk_offset(2, p, lane >> 1) + (lane & 1) * 8) = vv;
+        }
     } else {
         const uint4 kk = *reinterpret_cast<const uint4*>(static_cast<const float*>(k) + row);
         const uint4 vv = *reinterpret_cast<const uint4*>(static_cast<const float*>(v) + row);
         kraw[0] = kk.x; kraw[1] = kk.y; kraw[2] = kk.z; kraw[3] = kk.w;
-        vraw[0] = vv.x; vraw[1] = vv.y; vraw[2] = vv.z; vraw[3] = vv.w;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) kf[i] = __uint_as_float(kraw[i]);
+        if (L.keep_v < kHeadDim) { vraw[0] = vv.x; vraw[1] = vv.y; vraw[2] = vv.z; vraw[3] = vv.w; }
+        else *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(4, p, lane)) = vv;
     }
+    if (L.keep_v < kHeadDim) {                             // value-channel pruning: same selection on |V|
+        float vf[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) vf[i] = __uint_as_float(kBf16 ? vraw[i] << 16 : vraw[i]);
+        const float one[4] = {1.f, 1.f, 1.f, 1.f};
+        pack_token<kBf16>(image, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
+    }
+    pack_token<kBf16>(image, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -220,6 +217,7 @@ struct CompressArgs {
     int keep;
     int64_t n_pool_pages;
     PageLayout L;
+    double inv_pruned;            // 1 / (D - T), 0 when T = D
     int* status;
 };
 
@@ -248,9 +246,7 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
         const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
                             static_cast<int64_t>(src_t) * A.st + lane * 4;
-        unsigned kraw[4], vraw[4];
-        load_kv_row<kBf16>(A.k, A.v, row, kraw, vraw);
-        pack_token_kv<kBf16>(image, L, p, lane, a, kraw, vraw);
+        pack_token_kv<kBf16>(image, L, p, lane, a, A.k, A.v, row, A.inv_pruned);
     }
     __syncthreads();
 
@@ -280,6 +276,7 @@ struct AppendArgs {
     PageLayout L;
     const float* qnorm;
     int32_t* packed_lens;
+    double inv_pruned;            // 1 / (D - T), 0 when T = D
     int* status;
 };
 
@@ -308,9 +305,7 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
     const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
     const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
-    unsigned kraw[4], vraw[4];
-    load_kv_row<kBf16>(A.k_new, A.v_new, row, kraw, vraw);
-    pack_token_kv<kBf16>(page, L, p, lane, a, kraw, vraw);
+    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned);
 }
 
 __global__ void append_advance_kernel(AppendArgs A)
@@ -329,6 +324,7 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     A.k_new = k_new; A.v_new = v_new; A.pages = static_cast<unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.B = p.batch; A.Hkv = p.n_kv_heads; A.keep = p.keep; A.n_pool_pages = p.n_pool_pages;
     A.L = make_layout(p.dtype, p.keep, p.keep_v); A.qnorm = qnorm; A.packed_lens = packed_lens;
+    A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
     A.status = static_cast<int*>(workspace);
     const dim3 grid(p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16) append_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(A);
@@ -470,6 +466,7 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
     A.qnorm = qnorm; A.pages = static_cast<unsigned char*>(pages);
     A.block_table = block_table; A.max_blocks = max_blocks; A.Hkv = p.n_kv_heads; A.keep = p.keep;
     A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep, p.keep_v); A.status = status;
+    A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
     const dim3 grid(n_blocks, p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16)
         compress_pages_kernel<__nv_bfloat16><<<grid, 256, A.L.page_bytes, stream>>>(A);
