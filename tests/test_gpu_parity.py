@@ -156,6 +156,16 @@ def test_many_units_cross_cta_boundaries():
     check_case(wl, 64, check_vals=False)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_largest_batch_with_empty_and_one_page_sequences(dtype):
+    """1024 sequences (the most one call takes), lengths 0..33: empty ones, single tokens, page tails."""
+    rng = np.random.default_rng(1024)
+    lens = rng.integers(0, 34, size=1024).tolist()
+    lens[0], lens[1], lens[-1] = 0, 33, 0
+    wl = make(dtype, 1024, 2, 1, lens, 4, 38, seed=110, sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
+    check_case(wl, 38, check_vals=False)
+
+
 def test_config2_llama_32k_full():
     c = inputs.CONFIGS[1]
     wl = inputs.config_workload(1, device="cuda")
