@@ -363,8 +363,10 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
         const int n = round * NS + lane;
         bool pending = owner && n < n_total;
         const int cur0 = id0, cur1 = id1;
-        // next revolution's ids: loads in flight while this revolution is polled
-        producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
+        // next revolution's ids: the lookup waits for its block-table loads, so it runs before the poll
+        // (hidden behind the wait for free slots) except in the first revolution, where every slot is
+        // free and the copies go out first
+        if (round > 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
         unsigned it = 0;
         while (__any_sync(kFull, pending)) {
             if (pending && (round == 0 || mbar_try_wait(empty, (round - 1) & 1))) {
@@ -381,6 +383,7 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
             if (++it >= kSpinLimit || *C.abort_flag) { live = false; break; }
         }
         if (!live) break;
+        if (round == 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
     }
     if (!live) {
         if (lane == 0) { *C.abort_flag = 1; record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT); }
