@@ -129,6 +129,23 @@ def test_single_token_and_empty_sequence():
     check_case(wl, 64)
 
 
+def test_all_sequences_empty():
+    wl = make("bf16", 2, 8, 2, [0, 0], 4, 64, seed=71, gap=False)
+    Bn, Hq, Hkv, W, D, S = wl.shape
+    cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=64, dtype="bf16", max_tokens=16)
+    cache.compress(wl.q_win, wl.k[:, :, :0].contiguous() if S == 0 else wl.k, wl.v, wl.seq_lens)
+    lse = torch.full((Bn, Hq), 1.0, dtype=torch.float32, device="cuda")
+    out = cache.decode(wl.q, out=torch.full((Bn, Hq, 128), 7.0, dtype=torch.float32, device="cuda"), lse=lse)
+    assert cache.status() == 0
+    assert bool((out == 0).all()) and bool(torch.isneginf(lse).all())
+
+
+@pytest.mark.parametrize("W", [1, 64])
+def test_window_sizes(W):
+    wl = make("bf16", 2, 8, 2, [70, 200], W, 38, seed=72 + W)
+    check_case(wl, 38)
+
+
 def test_paged_pool_with_permuted_block_table_qwen_shape():
     lens = [700, 33, 1200, 16]
     wl = make("bf16", 4, 28, 4, lens, 32, 38, seed=80)
