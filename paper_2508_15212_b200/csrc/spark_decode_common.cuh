@@ -198,12 +198,16 @@ __device__ __forceinline__ Segment locate(const int* prefix, int B, int Hkv, int
 //   aligned mode: all units have the same number of steps and there are several CTAs per unit; unit u
 //                 gets q or q+1 whole CTAs (the first `rem` units get q+1) and is split evenly among
 //                 them, so no CTA crosses a unit boundary and every CTA publishes exactly once.
+//   whole units : all units have the same number of steps and there are more units than CTAs; every CTA
+//                 takes q or q+1 whole units (the first `rem` CTAs take q+1).  No unit is split, so
+//                 there are no partials and no last-arriver merge; used when the uneven deal costs at
+//                 most 25 % over the even split.
 struct Plan {
     int total;        // steps on the line
     int chunk;        // stream mode: steps per CTA
-    int aligned;      // 1: aligned mode
-    int unit_steps;   // aligned mode: steps of every unit
-    int q, rem;       // aligned mode: CTAs per unit
+    int aligned;      // 0: stream, 1: aligned mode, 2: whole units
+    int unit_steps;   // aligned / whole units: steps of every unit
+    int q, rem;       // aligned: CTAs per unit; whole units: units per CTA
 };
 
 struct Ctrl {
@@ -282,6 +286,12 @@ __device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl&
                 if (q >= 2 && makespan * 25 <= pl.chunk * 26) {          // within 4 % of the even split
                     pl.aligned = 1; pl.q = q; pl.rem = nct - q * units;
                 }
+            } else if (smin == smax && smax > 0) {
+                const int q = units / nct, rem = units - q * nct;
+                const int makespan = (q + (rem ? 1 : 0)) * smax;
+                if (makespan * 4 <= pl.chunk * 5) {                      // within 25 % of the even split
+                    pl.aligned = 2; pl.q = q; pl.rem = rem;
+                }
             }
             *C.plan = pl;
         }
@@ -295,6 +305,12 @@ __device__ __forceinline__ void cta_range(const Plan& pl, int cta, int& c0, int&
     if (!pl.aligned) {
         c0 = min(pl.total, cta * pl.chunk);
         c1 = min(pl.total, c0 + pl.chunk);
+        return;
+    }
+    if (pl.aligned == 2) {                                  // whole units: the first `rem` CTAs take q + 1
+        const int first = cta * pl.q + min(cta, pl.rem);
+        c0 = first * pl.unit_steps;
+        c1 = c0 + (pl.q + (cta < pl.rem ? 1 : 0)) * pl.unit_steps;
         return;
     }
     const int big = pl.rem * (pl.q + 1);                   // CTAs that belong to units with q+1 CTAs
@@ -312,6 +328,12 @@ __device__ __forceinline__ void unit_parts(const Plan& pl, int unit_start, int u
     if (!pl.aligned) {
         first_cta = unit_start / pl.chunk;
         n_parts = (unit_start + unit_steps - 1) / pl.chunk - first_cta + 1;
+        return;
+    }
+    if (pl.aligned == 2) {
+        const int u2 = unit_start / pl.unit_steps, big = pl.rem * (pl.q + 1);
+        first_cta = u2 < big ? u2 / (pl.q + 1) : pl.rem + (u2 - big) / pl.q;
+        n_parts = 1;
         return;
     }
     const int u = unit_start / pl.unit_steps;

@@ -183,6 +183,13 @@ def test_largest_batch_with_empty_and_one_page_sequences(dtype):
     check_case(wl, 38, check_vals=False)
 
 
+@pytest.mark.parametrize("Bn,Hkv,n", [(37, 8, 150), (145, 2, 70)])
+def test_more_equal_units_than_ctas_whole_units_per_cta(Bn, Hkv, n):
+    """296 and 290 equal-length units on 148 CTAs: every CTA takes two whole units (or two and one)."""
+    wl = make("bf16", Bn, 2 * Hkv, Hkv, [n] * Bn, 8, 64, seed=120 + Bn, gap=False)
+    check_case(wl, 64, check_vals=False)
+
+
 def test_config2_llama_32k_full():
     c = inputs.CONFIGS[1]
     wl = inputs.config_workload(1, device="cuda")
