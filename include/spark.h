@@ -156,7 +156,8 @@ spark_status spark_compress(const spark_params *p,
  * value are concatenated to the cache, K <- Cat[K, k]).  The paper prunes during prefill and does not say
  * how keys appended later are treated; here the new key is pruned at once with the sequence's prefill
  * statistics: w[j] = qnorm[j] * |k[j]|, the `keep` largest channels are kept, mu is the mean of the rest --
- * exactly what spark_compress would have stored for that token given the same window queries.
+ * exactly what spark_compress would have stored for that token given the same window queries.  With
+ * value-channel pruning (keep_v) the new value row is pruned by |v[j]| in the same way.
  *
  *   k_new, v_new   [B][Hkv][D] contiguous, dtype as the cache, 16-byte aligned
  *   pages, block_table, max_blocks, qnorm   as used by spark_compress / spark_decode_attn; the page that
