@@ -129,7 +129,7 @@ def workload_desc(cfg, keep, copies=None, keep_v=0):
 def run_reference(args, cfg, keep):
     """The oracle as the reference arm: a bounded sample (one full decode step per timed step)."""
     import torch
-    from paper_2508_15212_b200 import inputs
+    from workloads import inputs
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -176,7 +176,8 @@ def main():
     args = ap.parse_args()
 
     import torch
-    from paper_2508_15212_b200 import inputs
+    from workloads import inputs
+    from paper_2508_15212_b200 import binding as B
     cfg = dict(inputs.CONFIGS[args.config])
     ratio = cfg["ratio"] if not isinstance(cfg["ratio"], tuple) else cfg["ratio"][1]
     if args.ratio is not None:
@@ -184,8 +185,8 @@ def main():
     if args.batch:
         cfg["batch"] = args.batch
     cfg["ratio"] = ratio
-    keep = args.keep or inputs.keep_count(cfg["head_dim"], ratio)
-    keep_v = inputs.keep_count(cfg["head_dim"], args.ratio_v) if args.ratio_v is not None else 0
+    keep = args.keep or B.spark_keep_count(cfg["head_dim"], ratio)
+    keep_v = B.spark_keep_count(cfg["head_dim"], args.ratio_v) if args.ratio_v is not None else 0
     if isinstance(cfg["seq_lens"], tuple):
         cfg["seq_lens"] = list(cfg["seq_lens"])
 
@@ -193,7 +194,6 @@ def main():
         run_reference(args, cfg, keep)
         return
 
-    from paper_2508_15212_b200 import binding as B
     from paper_2508_15212_b200 import build as spark_build
     from paper_2508_15212_b200.cache import SparkCache
 
@@ -212,7 +212,7 @@ def main():
     # ---- workload (weak scaling: every rank holds its own copy of the configuration) ----
     # A step is a list of (cache, q, out) decode launches: one for the single-layer configurations
     # (rotating over cold copies), 28 (one per layer) for the Qwen-shaped configuration.
-    from paper_2508_15212_b200.cache import build_evicted_batch, permuted_block_table
+    from workloads.batches import build_evicted_batch, permuted_block_table
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
     flags = 0 if args.no_overlap else B.SPARK_FLAG_OVERLAP_PREVIOUS
     D = cfg["head_dim"]

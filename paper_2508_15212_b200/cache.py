@@ -8,6 +8,8 @@ import torch
 from . import binding as B
 
 _TDT = {"f32": torch.float32, "bf16": torch.bfloat16}
+GUARD_BYTES = 4096          # canary band on each side of a guarded buffer
+GUARD_VALUE = 0xA5
 
 
 class SparkCache:
@@ -21,8 +23,10 @@ class SparkCache:
                  max_tokens: int, device="cuda", block_table: Optional[torch.Tensor] = None,
                  n_pool_pages: Optional[int] = None, token_budget: int = 0, pool_kernel: int = 7,
                  softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None, flags: int = 0,
-                 keep_v: int = 0):
+                 keep_v: int = 0, guard: bool = False):
         self.device = torch.device(device)
+        self.guard = bool(guard)          # debugging aid: canary bands around every buffer the library writes
+        self._bands = []                  # (name, raw uint8 tensor, payload bytes)
         self.dtype = dtype
         self.max_src_tokens = int(max_tokens)
         packed_max = min(max_tokens, token_budget) if token_budget > 0 else max_tokens
@@ -41,17 +45,45 @@ class SparkCache:
                                     softmax_scale=softmax_scale, flags=flags, keep_v=keep_v)
         self.page_bytes = B.spark_page_bytes(self.params)
         assert self.page_bytes > 0
-        self.pages = pages if pages is not None else torch.zeros(n_pool_pages * self.page_bytes,
-                                                                   dtype=torch.uint8, device=self.device)
-        self.qnorm = torch.empty(batch, n_kv_heads, 128, dtype=torch.float32, device=self.device)
-        self.packed_lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
-        self.kept_tokens = (torch.empty(batch, n_kv_heads, token_budget, dtype=torch.int32, device=self.device)
-                            if token_budget > 0 else None)
+        self.pages = pages if pages is not None else self._alloc("pages", n_pool_pages * self.page_bytes, zero=True)
+        self.qnorm = self._alloc("qnorm", batch * n_kv_heads * 128 * 4).view(torch.float32).view(batch, n_kv_heads, 128)
+        self.packed_lens = self._alloc("packed_lens", batch * 4, zero=True).view(torch.int32)
+        self.kept_tokens = (self._alloc("kept_tokens", batch * n_kv_heads * token_budget * 4).view(torch.int32)
+                            .view(batch, n_kv_heads, token_budget) if token_budget > 0 else None)
         cb, db = B.spark_workspace_bytes(self.params, self.max_src_tokens)
-        self.ws_compress = torch.empty(cb, dtype=torch.uint8, device=self.device)
-        self.ws_decode = torch.empty(db, dtype=torch.uint8, device=self.device)
+        self.ws_compress = self._alloc("ws_compress", cb)
+        self.ws_decode = self._alloc("ws_decode", db)
         B.spark_workspace_init(self.ws_compress)
         B.spark_workspace_init(self.ws_decode)
+
+    # -- buffers ----------------------------------------------------------------------------------
+    def _alloc(self, name: str, nbytes: int, zero: bool = False) -> torch.Tensor:
+        """A uint8 device buffer of `nbytes`; with guard=True it sits between two canary bands."""
+        if not self.guard:
+            return (torch.zeros if zero else torch.empty)(nbytes, dtype=torch.uint8, device=self.device)
+        raw = torch.full((nbytes + 2 * GUARD_BYTES,), GUARD_VALUE, dtype=torch.uint8, device=self.device)
+        payload = raw[GUARD_BYTES:GUARD_BYTES + nbytes]
+        if zero:
+            payload.zero_()
+        self._bands.append((name, raw, nbytes))
+        return payload
+
+    def alloc_out(self) -> torch.Tensor:
+        p = self.params
+        return self._alloc("out", p.batch * p.n_q_heads * 128 * 4).view(torch.float32).view(p.batch, p.n_q_heads, 128)
+
+    def alloc_lse(self) -> torch.Tensor:
+        p = self.params
+        return self._alloc("lse", p.batch * p.n_q_heads * 4).view(torch.float32).view(p.batch, p.n_q_heads)
+
+    def broken_guards(self):
+        """Names of guarded buffers whose canary bands were written to (empty list: all intact)."""
+        bad = []
+        for name, raw, nbytes in self._bands:
+            head, tail = raw[:GUARD_BYTES], raw[GUARD_BYTES + nbytes:]
+            if not (bool((head == GUARD_VALUE).all()) and bool((tail == GUARD_VALUE).all())):
+                bad.append(name)
+        return bad
 
     # -- the two calls of the method ------------------------------------------------------------
     def compress(self, q_win, k, v, seq_lens) -> None:
@@ -66,7 +98,7 @@ class SparkCache:
     def decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
         p = self.params
         if out is None:
-            out = torch.empty(p.batch, p.n_q_heads, 128, dtype=torch.float32, device=self.device)
+            out = self.alloc_out()
         B.spark_decode_attn(p, q, self.pages, self.block_table, self.packed_lens, self.qnorm, out, lse,
                             self.ws_decode)
         return out
@@ -95,64 +127,3 @@ class SparkCache:
     @property
     def algorithmic_bytes_per_token(self) -> int:
         return B.spark_algorithmic_bytes_per_token(self.params)
-
-
-# ---------------------------------------------------------------------------------------------------
-# Packed caches of the benchmark configurations (buffer plumbing; all arithmetic is in the library)
-# ---------------------------------------------------------------------------------------------------
-def permuted_block_table(batch: int, n_kv_heads: int, lens, device, seed: int, spare: int = 0):
-    """Block table of a paged pool: every (sequence, head) unit gets exactly the pages it needs, drawn
-    from a seeded random permutation of the pool.  Returns (table [B,Hkv,max_blocks] int32, n_pool_pages)."""
-    blocks = [(int(n) + 15) // 16 for n in lens]
-    max_blocks = max(max(blocks), 1)
-    n_pages = n_kv_heads * sum(blocks) + spare
-    g = torch.Generator().manual_seed(int(seed))
-    perm = torch.randperm(n_pages, generator=g).to(torch.int32)
-    table = torch.zeros(batch, n_kv_heads, max_blocks, dtype=torch.int32)
-    pos = 0
-    for b in range(batch):
-        for h in range(n_kv_heads):
-            table[b, h, :blocks[b]] = perm[pos:pos + blocks[b]]
-            pos += blocks[b]
-    return table.to(device), max(n_pages, 1)
-
-
-def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int = None, seed_offset: int = 0,
-                        keep_prompts: int = 0, flags: int = 0, keep_v: int = 0):
-    """Configuration 4: prompts are generated, evicted to the token budget and pruned ONE AT A TIME (each
-    prompt's dense K/V is freed before the next), into one shared page pool; the result is a batch cache
-    whose decode step serves all prompts.  Returns (cache, q [B,Hq,D], kept_tokens [B,Hkv,budget], dense)
-    where `dense` holds the first `keep_prompts` prompts' workloads for checks."""
-    from . import inputs
-    Bn = int(n_prompts or config["batch"])
-    Hq, Hkv, W, S = config["n_q_heads"], config["n_kv_heads"], config["window"], int(config["seq_lens"])
-    budget, pool = int(config["token_budget"]), int(config["pool_kernel"])
-    batch = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
-                       max_tokens=min(S, budget), device=device, flags=flags, keep_v=keep_v)
-    blocks = batch.max_blocks
-    qs, kept, dense = [], [], []
-    batch.prep_us = []                     # evict + prune time of each prompt (CUDA events)
-    for b in range(Bn):
-        wl = inputs.make_workload(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=S, window=W,
-                                  dtype=config["dtype"], sigma_s=config["sigma_s"],
-                                  seed=int(config["seed"]) + 7 * b + 1000003 * seed_offset, device=device)
-        one = SparkCache(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
-                         max_tokens=S, device=device, token_budget=budget, pool_kernel=pool,
-                         block_table=batch.block_table[b:b + 1].contiguous(),
-                         n_pool_pages=batch.params.n_pool_pages, pages=batch.pages, keep_v=keep_v)
-        assert one.block_table.shape[-1] == blocks
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        one.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
-        e1.record()
-        e1.synchronize()
-        batch.prep_us.append(e0.elapsed_time(e1) * 1e3)
-        batch.qnorm[b].copy_(one.qnorm[0])
-        batch.packed_lens[b:b + 1].copy_(one.packed_lens)
-        qs.append(wl.q[0])
-        kept.append(one.kept_tokens[0].clone())
-        assert one.status() == 0
-        if b < keep_prompts:
-            dense.append(wl)
-        del wl, one
-    return batch, torch.stack(qs), torch.stack(kept), dense

@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
             tc_stage_rows_async(k_u0 + static_cast<unsigned>((tile + 1 - tile0) & 1) * (kTcTile * 256u), kTcTile,
                                 k_unit + static_cast<int64_t>(t0 + kTcTile) * A.st, A.st,
                                 min(kTcTile, S - (t0 + kTcTile)), tid);
-        if (tid == 0) {
+        if (tid == 0 && !dead) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (PASS == 1) {
                 const unsigned idesc = tc_idesc(128, kTcTile);
@@ -223,13 +223,23 @@ __global__ void __launch_bounds__(kTcThreads, 2) evict_scores_tc_kernel(EvictTcA
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&mma_bar)) : "memory");
         }
-        // wait for the MMAs of this tile (bounded)
-        if (!dead) {
-            unsigned ok = 0;
+        // wait for the MMAs of this tile (bounded).  The verdict is made CTA-uniform by the barrier below, so
+        // that the warp-collective tensor-memory loads of the epilogue are never executed divergently and,
+        // once a wait has run out, no thread issues further MMAs or reads the accumulator.
+        {
+            unsigned ok = dead ? 1u : 0u;
             for (unsigned it = 0; it < kTcSpin && !ok; ++it)
                 asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                              : "=r"(ok) : "r"(tc_smem_u32(&mma_bar)), "r"(phase) : "memory");
-            if (!ok) { dead = true; record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT); }
+            const bool timed_out = __syncthreads_or(!ok) != 0;
+            if (timed_out && !dead) {
+                dead = true;
+                if (tid == 0) record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT);
+                // give the MMAs that were issued one more bounded chance to retire before the accumulator is freed
+                for (unsigned it = 0; it < kTcSpin && !ok; ++it)
+                    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                                 : "=r"(ok) : "r"(tc_smem_u32(&mma_bar)), "r"(phase) : "memory");
+            }
         }
         phase ^= 1u;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

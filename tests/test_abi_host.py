@@ -103,3 +103,33 @@ def test_null_and_shape_errors_come_before_any_launch(lib):
     assert lib.spark_read_status(null, null) == 1
     assert lib.spark_workspace_init(null, 1024, null) == 1
     assert B.spark_version() >= 100
+
+
+def test_misaligned_pointers_and_oversized_tables_are_refused_on_the_host(lib):
+    """q, qnorm and out are accessed with 16-byte vector loads / stores: a pointer that is not 16-byte aligned
+    would fault on the device, so it is turned away here.  16 * max_blocks must fit a 32-bit int."""
+    p = params()
+    null, one, ws = ctypes.c_void_p(None), ctypes.c_void_p(4096), ctypes.c_void_p(8192)
+    off8, off4 = ctypes.c_void_p(4096 + 8), ctypes.c_void_p(4096 + 4)
+
+    def decode(q=one, qnorm=one, out=one, lse=null, max_blocks=4):
+        return lib.spark_decode_attn(ctypes.byref(p), q, one, one, max_blocks, one, qnorm, out, lse, ws, 1 << 30, null)
+
+    assert decode(q=off8) == 2 and decode(qnorm=off8) == 2 and decode(out=off4) == 2
+    assert decode(lse=ctypes.c_void_p(4096 + 2)) == 2
+    assert decode(max_blocks=(2 ** 31 - 1) // 16 + 1) == 2
+
+    def noalloc(q=one, qnorm=one, out=one, max_blocks=4):
+        return lib.spark_decode_attn_noalloc(ctypes.byref(p), q, one, one, max_blocks, one, qnorm, out, null, null)
+
+    assert noalloc(q=off8) == 2 and noalloc(qnorm=off8) == 2 and noalloc(out=off4) == 2
+    assert noalloc(max_blocks=(2 ** 31 - 1) // 16 + 1) == 2
+    # spark_compress writes qnorm and the page kernel reads it back four floats at a time
+    rc = lib.spark_compress(ctypes.byref(p), one, one, one, 0, 0, 128, one, 64, one, one, 4, off8, one, null,
+                            ws, 1 << 30, null)
+    assert rc == 2
+    rc = lib.spark_compress(ctypes.byref(p), one, one, one, 0, 0, 128, one, 64, one, one, (2 ** 31 - 1) // 16 + 1,
+                            one, one, null, ws, 1 << 30, null)
+    assert rc == 2
+    rc = lib.spark_append(ctypes.byref(p), one, one, one, one, 4, off8, one, ws, 1 << 20, null)
+    assert rc == 2

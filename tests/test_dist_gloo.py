@@ -5,7 +5,8 @@ import socket
 import torch
 import torch.multiprocessing as mp
 
-from paper_2508_15212_b200 import dist_utils, inputs
+from paper_2508_15212_b200 import dist_utils
+from workloads import inputs
 
 
 def _free_port():

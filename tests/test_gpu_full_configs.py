@@ -12,8 +12,9 @@ import torch
 import oracle
 from paper_2508_15212_b200 import binding as B
 from paper_2508_15212_b200 import build as spark_build
-from paper_2508_15212_b200 import inputs
-from paper_2508_15212_b200.cache import SparkCache, build_evicted_batch, permuted_block_table
+from paper_2508_15212_b200.cache import SparkCache
+from workloads import inputs
+from workloads.batches import build_evicted_batch, permuted_block_table
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-3          # bf16 storage, fp32 accumulation
@@ -63,7 +64,7 @@ def check_unit(wl, cache, out, b, h, keep, lens, keep_v=0):
 
 def test_config3_4x128k_ratio08_sampled_units():
     cfg = inputs.CONFIGS[2]
-    for keep in (inputs.keep_count(128, cfg["ratio"]), 26):        # floor rule (25) and the rounded count (26)
+    for keep in (B.spark_keep_count(128, cfg["ratio"]), 26):        # floor rule (25) and the rounded count (26)
         wl = inputs.config_workload(2, device="cuda")
         inputs.enforce_saliency_gap(wl, keep)
         Bn, Hq, Hkv, W, D, S = wl.shape
@@ -86,46 +87,53 @@ def test_config3_4x128k_ratio08_sampled_units():
 
 
 def test_config4_evicted_batch_pruning_and_decode():
+    """All 32 prompts, as benchmarked: 256 units of 2048 tokens on 148 CTAs, i.e. the whole-units plan with
+    two units in each of the first 108 CTAs and one in each of the remaining 40."""
     cfg = dict(inputs.CONFIGS[3])
-    keep = inputs.keep_count(128, cfg["ratio"])
-    n_prompts = 8                                                 # same path as the 32 of the benchmark
-    cache, q, kept, dense = build_evicted_batch(cfg, keep, n_prompts=n_prompts, keep_prompts=1)
+    keep = B.spark_keep_count(128, cfg["ratio"])
+    n_prompts = cfg["batch"]
+    assert n_prompts == 32
+    cache, q, kept, dense = build_evicted_batch(cfg, keep, n_prompts=n_prompts, keep_prompts=(0, 27, 31), guard=True)
     Hq, Hkv, W, budget, S = cfg["n_q_heads"], cfg["n_kv_heads"], cfg["window"], cfg["token_budget"], cfg["seq_lens"]
     G = Hq // Hkv
     assert cache.packed_lens.cpu().tolist() == [budget] * n_prompts
     kept_np = kept.cpu().numpy()
     assert (np.diff(kept_np, axis=-1) > 0).all() and (kept_np[..., -W:] == np.arange(S - W, S)).all()
     out = cache.decode(q)
-    assert cache.status() == 0
+    assert cache.status() == 0 and cache.broken_guards() == []
     u = cache.unpack(want_vals=False, want_v=False)
     assert bool((popcounts(u["mask"]) == keep).all())
-    # eviction against the oracle on sampled units of prompt 0 (the oracle needs ~4 GFLOP per unit)
-    wl = dense[0]
-    for h in (0, 5):
+    # units (0,0) and (0,1) are the first and second unit of CTA 0; (0,5) sits in CTA 2; units of prompts 27..31
+    # (unit index >= 216) are alone in their CTA
+    checks = [(0, 0, True), (0, 1, False), (0, 5, True), (27, 3, True), (31, 7, False)]
+    for b, h, with_eviction in checks:
+        wl = dense[b]
         q_win = wl.q_win[:, h * G:(h + 1) * G].cpu()
-        k = wl.k[:, h:h + 1].cpu().contiguous()
-        ref_kept, n, vote, pooled = oracle.evict(q_win, k, [S], budget, cfg["pool_kernel"], want_votes=True)
-        srt = np.sort(pooled[0, 0, :S - W])[::-1]
-        gap = (srt[budget - W - 1] - srt[budget - W]) / srt[budget - W - 1]
-        same = np.array_equal(kept_np[0, h], ref_kept[0, 0])
-        overlap = len(set(kept_np[0, h].tolist()) & set(ref_kept[0, 0].tolist()))
-        assert same or (gap <= 1e-4 and overlap >= budget - 2), f"head {h}: overlap {overlap}, gap {gap:.2e}"
+        if with_eviction:                                  # the oracle needs ~4 GFLOP per unit
+            k = wl.k[:, h:h + 1].cpu().contiguous()
+            ref_kept, n, vote, pooled = oracle.evict(q_win, k, [S], budget, cfg["pool_kernel"], want_votes=True)
+            srt = np.sort(pooled[0, 0, :S - W])[::-1]
+            gap = (srt[budget - W - 1] - srt[budget - W]) / srt[budget - W - 1]
+            same = np.array_equal(kept_np[b, h], ref_kept[0, 0])
+            overlap = len(set(kept_np[b, h].tolist()) & set(ref_kept[0, 0].tolist()))
+            assert same or (gap <= 1e-4 and overlap >= budget - 2), f"unit ({b},{h}): overlap {overlap}, gap {gap:.2e}"
         # pruning + decode of this unit on the evicted token set fed to both sides
-        idx = torch.from_numpy(kept_np[0, h].astype(np.int64))
+        idx = torch.from_numpy(kept_np[b, h].astype(np.int64))
         kg = wl.k[0, h].cpu()[idx].view(1, 1, budget, 128).contiguous()
         vg = wl.v[0, h].cpu()[idx].view(1, 1, budget, 128).contiguous()
         _, a = oracle.window_mean(q_win, 1)
+        assert np.array_equal(cache.qnorm[b, h].cpu().numpy(), a[0, 0])
         c = oracle.compress(kg, [budget], keep, a)
-        ref, _ = oracle.decode_attn(q[0:1, h * G:(h + 1) * G].cpu(), kg, vg, [budget], c["mask"], c["mu"], a)
-        assert np.array_equal(u["mask"][0, h].cpu().numpy().view(np.uint32), c["mask"][0, 0])
-        d = float(np.abs(out[0, h * G:(h + 1) * G].cpu().numpy() - ref[0]).max())
-        assert d <= TOL, f"head {h} max|delta| {d:.3e}"
+        ref, _ = oracle.decode_attn(q[b:b + 1, h * G:(h + 1) * G].cpu(), kg, vg, [budget], c["mask"], c["mu"], a)
+        assert np.array_equal(u["mask"][b, h].cpu().numpy().view(np.uint32), c["mask"][0, 0])
+        d = float(np.abs(out[b, h * G:(h + 1) * G].cpu().numpy() - ref[0]).max())
+        assert d <= TOL, f"unit ({b},{h}) max|delta| {d:.3e}"
 
 
 @pytest.mark.parametrize("ratio", [0.3, 0.5, 0.7, 0.8])
 def test_config5_qwen_paged_variable_lengths(ratio):
     cfg = inputs.CONFIGS[4]
-    keep = inputs.keep_count(128, ratio)
+    keep = B.spark_keep_count(128, ratio)
     for layer in (0, 27):
         wl = inputs.config_workload(4, device="cuda", seed_offset=layer)
         Bn, Hq, Hkv, W, D, S = wl.shape
@@ -162,7 +170,7 @@ def test_config5_qwen_paged_variable_lengths(ratio):
 
 def test_config5_qwen_paged_with_value_pruning():
     """Layer 0 of the Qwen-shaped configuration with (0.5 + 0.5) key + value channel pruning."""
-    keep = keep_v = inputs.keep_count(128, 0.5)
+    keep = keep_v = B.spark_keep_count(128, 0.5)
     wl = inputs.config_workload(4, device="cuda", seed_offset=0)
     Bn, Hq, Hkv, W, D, S = wl.shape
     lens = wl.seq_lens.tolist()

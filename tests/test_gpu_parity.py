@@ -10,7 +10,8 @@ import torch
 import oracle
 from paper_2508_15212_b200 import binding as B
 from paper_2508_15212_b200 import build as spark_build
-from paper_2508_15212_b200 import inputs
+from workloads import inputs
+from workloads.batches import permuted_block_table
 from paper_2508_15212_b200.cache import SparkCache
 
 pytestmark = pytest.mark.gpu
@@ -47,7 +48,7 @@ def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True, k
     wl_cpu = wl.to("cpu")
     a, c, o_ref, lse_ref = oracle_side(wl_cpu, keep, keep_v)
     cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
-                       max_tokens=S, block_table=block_table, n_pool_pages=n_pool_pages, keep_v=keep_v)
+                       max_tokens=S, block_table=block_table, n_pool_pages=n_pool_pages, keep_v=keep_v, guard=True)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     lens = wl_cpu.seq_lens.tolist()
     assert cache.packed_lens.cpu().tolist() == lens
@@ -75,11 +76,12 @@ def check_case(wl, keep, block_table=None, n_pool_pages=None, check_vals=True, k
             bits = (c["vmask"][..., None] >> np.arange(32, dtype=np.uint32)) & 1
             vv = np.where(bits.reshape(vv.shape).astype(bool), vv, np.zeros_like(vv))
         assert np.array_equal(to_np(u["v"]), vv)
-    lse = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
+    lse = cache.alloc_lse()
     out = cache.decode(wl.q, lse=lse)
     out2 = cache.decode(wl.q)                                    # tickets self-reset; result reproducible
     assert cache.status() == 0
     assert torch.equal(out, out2)
+    assert cache.broken_guards() == [], "a kernel wrote outside one of its buffers"
     d = float(np.abs(out.cpu().numpy() - o_ref).max())
     assert d <= TOL[wl.dtype], f"max|delta| {d:.3e} (max|out| {np.abs(o_ref).max():.3e})"
     l = lse.cpu().numpy()
@@ -209,8 +211,8 @@ def test_bad_page_id_is_recorded_not_dereferenced():
     assert B.spark_read_status(cache.ws_decode) == 6            # SPARK_ERR_DEVICE_BOUNDS
 
 
-def evicted_reference(wl_cpu, budget, pool, keep):
-    """Oracle side of eviction + pruning + decode: returns kept tokens, lengths, boundary gaps, output."""
+def oracle_evicted_sets(wl_cpu, budget, pool):
+    """Oracle eviction: kept tokens, lengths and the relative gap of the pooled votes at the budget boundary."""
     Bn, Hq, Hkv, W, D, S = wl_cpu.shape
     lens = wl_cpu.seq_lens.tolist()
     kept, n, vote, pooled = oracle.evict(wl_cpu.q_win, wl_cpu.k, lens, budget, pool, want_votes=True)
@@ -222,6 +224,13 @@ def evicted_reference(wl_cpu, budget, pool, keep):
         for h in range(Hkv):
             srt = np.sort(pooled[b, h, :P])[::-1]
             gaps[b, h] = (srt[k - 1] - srt[k]) / max(srt[k - 1], 1e-300)
+    return kept, n, gaps
+
+
+def oracle_on_kept_tokens(wl_cpu, kept, n, keep):
+    """Oracle pruning + decode over the tokens listed in `kept` ([B][Hkv][budget], first n[b] valid)."""
+    Bn, Hq, Hkv, W, D, S = wl_cpu.shape
+    budget = kept.shape[-1]
     kk, vv = to_np(wl_cpu.k), to_np(wl_cpu.v)
     kg, vg = np.zeros((Bn, Hkv, budget, D), kk.dtype), np.zeros((Bn, Hkv, budget, D), vv.dtype)
     for b in range(Bn):
@@ -232,24 +241,29 @@ def evicted_reference(wl_cpu, budget, pool, keep):
     _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
     c = oracle.compress(kg, n, keep, a)
     out, _ = oracle.decode_attn(to_np(wl_cpu.q), kg, vg, n, c["mask"], c["mu"], a)
-    return kept, n, gaps, c, out
+    return c, out, kg, vg
 
 
 @pytest.mark.parametrize("dtype,lens,W,budget,G", [("bf16", [600, 90, 300], 8, 128, 4),
                                                    ("bf16", [2000], 32, 256, 7),
                                                    ("f32", [500, 64], 16, 96, 2)])
 def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
+    """Three checks, none of them conditional on the other: (1) the evicted token sets against the oracle's
+    (exact where the pooled votes at the budget boundary are not a near-tie); (2) pruning and decode of the
+    evicting call against the oracle run on the SAME token set (the one the GPU kept); (3) pruning and decode
+    of the oracle's token set, gathered and fed to both sides through the non-evicting call.  A near-tie in
+    (1) can therefore never hide a pruning or decode error."""
     keep, Hkv, Bn = 64, 2, len(lens)
     wl = make(dtype, Bn, Hkv * G, Hkv, lens, W, keep, seed=130 + G, sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
     wl_cpu = wl.to("cpu")
-    kept_ref, n_ref, gaps, c_ref, out_ref = evicted_reference(wl_cpu, budget, 7, keep)
+    kept_ref, n_ref, gaps = oracle_evicted_sets(wl_cpu, budget, 7)
     cache = SparkCache(batch=Bn, n_q_heads=Hkv * G, n_kv_heads=Hkv, window=W, keep=keep, dtype=dtype,
-                       max_tokens=max(lens), token_budget=budget, pool_kernel=7)
+                       max_tokens=max(lens), token_budget=budget, pool_kernel=7, guard=True)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     assert cache.status() == 0
     assert cache.packed_lens.cpu().tolist() == n_ref.tolist()
     kept = cache.kept_tokens.cpu().numpy()
-    same = True
+    # (1) token sets
     for b in range(Bn):
         for h in range(Hkv):
             a_, r_ = kept[b, h, :n_ref[b]], kept_ref[b, h, :n_ref[b]]
@@ -257,15 +271,33 @@ def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
             if gaps[b, h] > 1e-4:
                 assert np.array_equal(a_, r_), f"evicted set differs at unit ({b},{h}), gap {gaps[b, h]:.2e}"
             else:
-                same = same and np.array_equal(a_, r_)
                 assert len(set(a_.tolist()) & set(r_.tolist())) >= n_ref[b] - 2
-    if same:
-        u = cache.unpack(want_vals=False, want_v=False)
-        assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c_ref["mask"])
-        out = cache.decode(wl.q)
-        assert cache.status() == 0
-        d = float(np.abs(out.cpu().numpy() - out_ref).max())
-        assert d <= TOL[dtype], f"max|delta| {d:.3e}"
+    # (2) the evicting call's pages and output against the oracle on the GPU's own token set
+    c_gpu, out_gpu_ref, _, _ = oracle_on_kept_tokens(wl_cpu, kept, n_ref, keep)
+    u = cache.unpack(want_vals=False, want_v=False)
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c_gpu["mask"])
+    assert np.allclose(u["mu"].cpu().numpy(), c_gpu["mu"], rtol=1e-6, atol=0)
+    out = cache.decode(wl.q)
+    assert cache.status() == 0
+    d = float(np.abs(out.cpu().numpy() - out_gpu_ref).max())
+    assert d <= TOL[dtype], f"evicting call: max|delta| {d:.3e}"
+    assert cache.broken_guards() == []
+    # (3) the oracle's token set, gathered, through the non-evicting call
+    c_ref, out_ref, kg, vg = oracle_on_kept_tokens(wl_cpu, kept_ref, n_ref, keep)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    as_t = (lambda x: torch.from_numpy(x.view(np.int16)).view(torch.bfloat16)) if dtype == "bf16" else torch.from_numpy
+    kg_t, vg_t = as_t(kg).cuda(), as_t(vg).cuda()
+    assert kg_t.dtype == tdt
+    plain = SparkCache(batch=Bn, n_q_heads=Hkv * G, n_kv_heads=Hkv, window=W, keep=keep, dtype=dtype,
+                       max_tokens=budget, guard=True)
+    plain.compress(wl.q_win, kg_t, vg_t, torch.from_numpy(n_ref).cuda())
+    u = plain.unpack(want_vals=False, want_v=False)
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c_ref["mask"])
+    out = plain.decode(wl.q)
+    assert plain.status() == 0
+    d = float(np.abs(out.cpu().numpy() - out_ref).max())
+    assert d <= TOL[dtype], f"oracle's token set: max|delta| {d:.3e}"
+    assert plain.broken_guards() == []
 
 
 def test_overlap_flag_gives_identical_results_back_to_back():
@@ -326,7 +358,6 @@ def test_value_pruning_bf16_ragged(keep, keep_v):
 def test_value_pruning_group_sizes_and_paged_pool(G, keep, keep_v):
     lens = [300, 47]
     wl = make("bf16", 2, 2 * G, 2, lens, 16, keep, seed=340 + G)
-    from paper_2508_15212_b200.cache import permuted_block_table
     table, n_pages = permuted_block_table(2, 2, lens, "cuda", seed=7, spare=3)
     check_case(wl, keep, block_table=table, n_pool_pages=n_pages, keep_v=keep_v)
 

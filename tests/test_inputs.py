@@ -1,9 +1,10 @@
 """The seeded generators: determinism, value structure, and the conditioning the benchmark asks for."""
+import math
 import numpy as np
 import torch
 
 import oracle
-from paper_2508_15212_b200 import inputs
+from workloads import inputs
 
 
 def small(seed=0, dtype="bf16", **kw):
@@ -49,4 +50,4 @@ def test_config_table_shapes():
     wl = inputs.config_workload(4, batch=3, seed_offset=1, seq_lens=[40, 17, 33])
     assert wl.shape[:5] == (3, 28, 4, 32, 128)
     c5 = inputs.config_workload.__globals__["CONFIGS"][4]
-    assert [inputs.keep_count(128, r) for r in c5["ratio"]] == [89, 64, 38, 25]
+    assert [int(math.floor((1.0 - r) * 128 + 1e-9)) for r in c5["ratio"]] == [89, 64, 38, 25]

@@ -278,8 +278,10 @@ def test_empty_sequence_gives_zero_output():
 
 def test_memory_accounting_of_kept_values():
     """Kept key values are T/D of the dense keys; at ratio 0.8 K+V values are 60 % (a 40 % cut)."""
-    from paper_2508_15212_b200.inputs import keep_count
     D = 128
+
+    def keep_count(d, lam):                                            # T = floor((1 - lambda) D)
+        return int(math.floor((1.0 - lam) * d + 1e-9))
     assert keep_count(D, 0.5) == 64 and keep_count(D, 0.8) == 25       # floor((1-lambda) D)
     assert keep_count(D, 0.3) == 89 and keep_count(D, 0.7) == 38 and keep_count(D, 0.0) == 128
     lam = 0.8
@@ -322,6 +324,62 @@ def test_eviction_pool_one_is_plain_top_k_of_causal_window_votes():
     _, _, vote5, pooled5 = oracle.evict(q_win, k, [S], budget=budget, pool=5, want_votes=True)
     for t in range(P):
         assert pooled5[0, 0, t] == vote5[0, 0, max(0, t - 2):min(P, t + 3)].max()
+
+
+def independent_votes(q_win, k, S, W, D):
+    """Causal observation-window votes of one KV head, written directly with NumPy (group summed)."""
+    P = S - W
+    vote = np.zeros(P)
+    for g in range(q_win.shape[0]):
+        for w in range(W):
+            last = P + w
+            s = k[:last + 1].astype(np.float64) @ q_win[g, w].astype(np.float64) / math.sqrt(D)
+            e = np.exp(s - s.max())
+            vote += (e / e.sum())[:P]
+    return vote
+
+
+@pytest.mark.parametrize("pool,S,W,budget,seed", [(7, 61, 4, 20, 16), (7, 200, 8, 40, 17), (3, 33, 2, 9, 18),
+                                                  (7, 12, 3, 6, 19)])
+def test_eviction_kept_set_is_top_k_of_the_POOLED_votes(pool, S, W, budget, seed):
+    """End to end at pool > 1: independent votes -> independent clamped max-pool -> top-(budget - W) with ties
+    to the lower position -> + window.  An oracle that ranked the raw votes would fail here."""
+    rng = np.random.default_rng(seed)
+    B, Hq, Hkv, D = 1, 4, 2, 16
+    q_win, k, v, q = rand_case(rng, B, Hq, Hkv, W, D, S)
+    kept, n = oracle.evict(q_win, k, [S], budget=budget, pool=pool)
+    assert n[0] == budget
+    P, half, G = S - W, (pool - 1) // 2, Hq // Hkv
+    differs_from_raw_ranking = False
+    for h in range(Hkv):
+        vote = independent_votes(q_win[0, h * G:(h + 1) * G], k[0, h], S, W, D)
+        pooled = np.array([vote[max(0, t - half):min(P, t + half + 1)].max() for t in range(P)])
+        order = sorted(range(P), key=lambda t: (-pooled[t], t))
+        want = sorted(order[:budget - W]) + list(range(P, S))
+        assert list(kept[0, h]) == want
+        # max-pooling makes equal pooled values routine: the boundary of this case must cut through a tie
+        # group somewhere in the sweep, which exercises the lower-position rule
+        raw = sorted(sorted(range(P), key=lambda t: (-vote[t], t))[:budget - W]) + list(range(P, S))
+        differs_from_raw_ranking |= (raw != want)
+    assert differs_from_raw_ranking, "case too weak: pooled and raw rankings keep the same tokens"
+
+
+def test_eviction_boundary_inside_a_run_of_equal_pooled_values():
+    """One dominant key makes `pool` neighbours share the same pooled value; a budget that ends inside that
+    run must keep the LOWER positions of the run."""
+    B, Hq, Hkv, W, D, S, pool = 1, 1, 1, 2, 8, 30, 7
+    rng = np.random.default_rng(20)
+    q_win = rng.standard_normal((B, Hq, W, D)).astype(np.float32)
+    k = (0.01 * rng.standard_normal((B, Hkv, S, D))).astype(np.float32)
+    k[0, 0, 15] = 4.0 * q_win[0, 0].mean(axis=0)                       # token 15 takes nearly all attention
+    P = S - W
+    vote = independent_votes(q_win[0], k[0, 0], S, W, D)
+    pooled = np.array([vote[max(0, t - 3):min(P, t + 4)].max() for t in range(P)])
+    run = [t for t in range(P) if pooled[t] == pooled[15]]
+    assert run == list(range(12, 19))                                  # the 7-neighbourhood of the dominant token
+    for extra in range(1, 7):                                          # budget ends inside the run
+        kept, n = oracle.evict(q_win, k, [S], budget=W + extra, pool=pool)
+        assert list(kept[0, 0]) == run[:extra] + list(range(P, S))
 
 
 # ---------------------------------------------------------------- value-channel pruning (App. "Pruning Value Cache Channels")

@@ -2,17 +2,20 @@
 
 spark_decode_attn_noalloc serves callers that are handed device tensors but may not allocate (no
 workspace to pass): it runs the same kernels on a scratch array built into the library.  The check: on
-the same packed cache its output equals the regular entry point's (same tolerance as the parity tests),
-on two calls in a row (the second call finds the scratch as the first left it), and problems beyond the
-built-in scratch are refused before anything is launched.  Collected last on purpose.
+the same packed cache its output equals the regular entry point's AND the CPU oracle's (same tolerance as
+the parity tests), on two calls in a row (the second call finds the scratch as the first left it), and
+problems beyond the built-in scratch are refused before anything is launched.  Collected last on purpose.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle
+
 from paper_2508_15212_b200 import binding as B
 from paper_2508_15212_b200 import build as spark_build
-from paper_2508_15212_b200 import inputs
 from paper_2508_15212_b200.cache import SparkCache
+from workloads import inputs
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +43,12 @@ def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, kee
     lse_ref = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
     ref = cache.decode(wl.q, lse=lse_ref)
     assert cache.status() == 0
+    # the oracle on the same inputs: an error common to both entry points cannot pass
+    wl_cpu = wl.to("cpu")
+    _, a = oracle.window_mean(wl_cpu.q_win, Hkv)
+    c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a)
+    vm = oracle.prune_values(wl_cpu.v, wl_cpu.seq_lens, keep_v) if 0 < keep_v < 128 else None
+    o_ref, l_ref = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, c["mask"], c["mu"], a, vmask=vm)
     for call in range(2):
         out = torch.full((Bn, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
         lse = torch.full((Bn, Hq), float("nan"), dtype=torch.float32, device="cuda")
@@ -49,6 +58,9 @@ def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, kee
         d = float((out - ref).abs().max())
         assert d <= TOL[dtype], f"call {call}: max|delta| {d:.3e}"
         assert float((lse - lse_ref).abs().max()) <= 1e-3
+        d = float(np.abs(out.cpu().numpy() - o_ref).max())
+        assert d <= TOL[dtype], f"call {call}: max|delta| vs oracle {d:.3e}"
+        assert float(np.abs(lse.cpu().numpy() - l_ref).max()) <= (1e-3 if dtype == "bf16" else 2e-5)
 
 
 def test_noalloc_refuses_problems_beyond_its_scratch():

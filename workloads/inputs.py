@@ -171,12 +171,6 @@ def enforce_saliency_gap(wl: Workload, keep: int, rel_gap: float = 2.0 ** -6,
 # The benchmark configurations (shapes, lengths and value structure of BASELINE configs).
 # --------------------------------------------------------------------------------------
 
-def keep_count(head_dim: int, ratio: float) -> int:
-    """T = floor((1 - ratio) * D), guarded against binary representation error."""
-    import math
-    return int(math.floor((1.0 - ratio) * head_dim + 1e-9))
-
-
 CONFIGS: List[Dict[str, object]] = [
     dict(name="tiny_fp32", batch=1, n_q_heads=1, n_kv_heads=1, head_dim=128, seq_lens=1024,
          window=32, dtype="f32", sigma_s=0.5, ratio=0.5, seed=0),
