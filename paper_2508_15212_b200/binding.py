@@ -95,6 +95,14 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
+def _blocks(block_table, max_blocks) -> int:
+    """Table width: the table's last dimension, or `max_blocks` for a contiguous cache (no table)."""
+    if block_table is not None:
+        return int(block_table.shape[-1])
+    assert max_blocks is not None, "a contiguous cache (block_table=None) needs max_blocks"
+    return int(max_blocks)
+
+
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
@@ -142,49 +150,53 @@ def spark_workspace_init(workspace: torch.Tensor) -> None:
 
 
 def spark_compress(p: spark_params, q_win, k, v, seq_lens, max_seq_tokens, pages, block_table, qnorm,
-                   packed_lens, kept_tokens, workspace) -> None:
+                   packed_lens, kept_tokens, workspace, max_blocks=None) -> None:
     assert k.stride(-1) == 1 and v.stride() == k.stride() and q_win.is_contiguous()
     sb, sh, st = k.stride(0), k.stride(1), k.stride(2)
     _check(lib().spark_compress(ctypes.byref(p), _ptr(q_win), _ptr(k), _ptr(v), sb, sh, st, _ptr(seq_lens),
-                                int(max_seq_tokens), _ptr(pages), _ptr(block_table), block_table.shape[-1],
+                                int(max_seq_tokens), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
                                 _ptr(qnorm), _ptr(packed_lens), _ptr(kept_tokens), _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _stream()),
            "spark_compress")
 
 
-def spark_append(p: spark_params, k_new, v_new, pages, block_table, qnorm, packed_lens, workspace) -> None:
+def spark_append(p: spark_params, k_new, v_new, pages, block_table, qnorm, packed_lens, workspace,
+                 max_blocks=None) -> None:
     assert k_new.is_contiguous() and v_new.is_contiguous()
     _check(lib().spark_append(ctypes.byref(p), _ptr(k_new), _ptr(v_new), _ptr(pages), _ptr(block_table),
-                              block_table.shape[-1], _ptr(qnorm), _ptr(packed_lens), _ptr(workspace),
+                              _blocks(block_table, max_blocks), _ptr(qnorm), _ptr(packed_lens), _ptr(workspace),
                               workspace.numel() * workspace.element_size(), _stream()),
            "spark_append")
 
 
-def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse, workspace) -> None:
+def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse, workspace,
+                      max_blocks=None) -> None:
     _check(lib().spark_decode_attn(ctypes.byref(p), _ptr(q), _ptr(pages), _ptr(block_table),
-                                   block_table.shape[-1], _ptr(packed_lens), _ptr(qnorm), _ptr(out), _ptr(lse),
+                                   _blocks(block_table, max_blocks), _ptr(packed_lens), _ptr(qnorm), _ptr(out), _ptr(lse),
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
            "spark_decode_attn")
 
 
-def spark_decode_attn_noalloc(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse) -> None:
+def spark_decode_attn_noalloc(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse,
+                              max_blocks=None) -> None:
     """Decode step that brings its own fixed scratch (batch * n_kv_heads <= 64); allocates nothing."""
     _check(lib().spark_decode_attn_noalloc(ctypes.byref(p), _ptr(q), _ptr(pages), _ptr(block_table),
-                                           block_table.shape[-1], _ptr(packed_lens), _ptr(qnorm), _ptr(out),
+                                           _blocks(block_table, max_blocks), _ptr(packed_lens), _ptr(qnorm), _ptr(out),
                                            _ptr(lse), _stream()),
            "spark_decode_attn_noalloc")
 
 
 def spark_unpack_pages(p: spark_params, pages, block_table, packed_lens, max_tokens, mask=None, mu=None,
-                       vals=None, v=None) -> None:
-    _check(lib().spark_unpack_pages(ctypes.byref(p), _ptr(pages), _ptr(block_table), block_table.shape[-1],
+                       vals=None, v=None, max_blocks=None) -> None:
+    _check(lib().spark_unpack_pages(ctypes.byref(p), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
                                     _ptr(packed_lens), int(max_tokens), _ptr(mask), _ptr(mu), _ptr(vals),
                                     _ptr(v), _stream()),
            "spark_unpack_pages")
 
 
-def spark_unpack_value_masks(p: spark_params, pages, block_table, packed_lens, max_tokens, vmask) -> None:
-    _check(lib().spark_unpack_value_masks(ctypes.byref(p), _ptr(pages), _ptr(block_table), block_table.shape[-1],
+def spark_unpack_value_masks(p: spark_params, pages, block_table, packed_lens, max_tokens, vmask,
+                             max_blocks=None) -> None:
+    _check(lib().spark_unpack_value_masks(ctypes.byref(p), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
                                           _ptr(packed_lens), int(max_tokens), _ptr(vmask), _stream()),
            "spark_unpack_value_masks")
 

@@ -15,8 +15,9 @@ GUARD_VALUE = 0xA5
 class SparkCache:
     """Owns the page pool, block table, qnorm, lens and workspaces for B sequences.
 
-    ``block_table`` defaults to the identity (contiguous cache); pass a permuted
-    table for a paged pool.  All arithmetic happens inside the library.
+    Without a ``block_table`` the cache is contiguous (the library is given no table: unit (b, h) owns
+    ``max_blocks`` consecutive pages); pass a table for a paged pool.  All arithmetic happens inside the
+    library.
     """
 
     def __init__(self, *, batch: int, n_q_heads: int, n_kv_heads: int, window: int, keep: int, dtype: str,
@@ -33,12 +34,15 @@ class SparkCache:
         self.max_tokens = int(packed_max)
         self.max_blocks = max(1, (self.max_tokens + 15) // 16)
         if block_table is None:
-            block_table = B.identity_block_table(batch, n_kv_heads, self.max_blocks, self.device)
-        self.block_table = block_table.to(self.device, torch.int32).contiguous()
-        assert self.block_table.shape == (batch, n_kv_heads, self.block_table.shape[-1])
-        assert self.block_table.shape[-1] >= self.max_blocks
+            self.block_table = None                       # contiguous cache: the calls get a NULL table
+            self.table_blocks = self.max_blocks
+        else:
+            self.block_table = block_table.to(self.device, torch.int32).contiguous()
+            assert self.block_table.shape == (batch, n_kv_heads, self.block_table.shape[-1])
+            assert self.block_table.shape[-1] >= self.max_blocks
+            self.table_blocks = int(self.block_table.shape[-1])
         if n_pool_pages is None:
-            n_pool_pages = batch * n_kv_heads * self.block_table.shape[-1]
+            n_pool_pages = batch * n_kv_heads * self.table_blocks
         self.params = B.make_params(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window,
                                     keep=keep, dtype=_TDT[dtype], n_pool_pages=n_pool_pages,
                                     token_budget=token_budget, pool_kernel=pool_kernel,
@@ -88,19 +92,19 @@ class SparkCache:
     # -- the two calls of the method ------------------------------------------------------------
     def compress(self, q_win, k, v, seq_lens) -> None:
         B.spark_compress(self.params, q_win, k, v, seq_lens, self.max_src_tokens, self.pages, self.block_table,
-                         self.qnorm, self.packed_lens, self.kept_tokens, self.ws_compress)
+                         self.qnorm, self.packed_lens, self.kept_tokens, self.ws_compress, max_blocks=self.table_blocks)
 
     def append(self, k_new, v_new) -> None:
         """One new token per sequence ([B, Hkv, D]), pruned with the prefill statistics."""
         B.spark_append(self.params, k_new, v_new, self.pages, self.block_table, self.qnorm, self.packed_lens,
-                       self.ws_compress)
+                       self.ws_compress, max_blocks=self.table_blocks)
 
     def decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
         p = self.params
         if out is None:
             out = self.alloc_out()
         B.spark_decode_attn(p, q, self.pages, self.block_table, self.packed_lens, self.qnorm, out, lse,
-                            self.ws_decode)
+                            self.ws_decode, max_blocks=self.table_blocks)
         return out
 
     # -- inspection ------------------------------------------------------------------------------
@@ -114,10 +118,11 @@ class SparkCache:
         if want_v:
             out["v"] = torch.empty(p.batch, p.n_kv_heads, n, 128, dtype=tdt, device=self.device)
         B.spark_unpack_pages(p, self.pages, self.block_table, self.packed_lens, n, out["mask"], out["mu"],
-                             out.get("vals"), out.get("v"))
+                             out.get("vals"), out.get("v"), max_blocks=self.table_blocks)
         if want_vmask:
             out["vmask"] = torch.empty(p.batch, p.n_kv_heads, n, 4, dtype=torch.int32, device=self.device)
-            B.spark_unpack_value_masks(p, self.pages, self.block_table, self.packed_lens, n, out["vmask"])
+            B.spark_unpack_value_masks(p, self.pages, self.block_table, self.packed_lens, n, out["vmask"],
+                                       max_blocks=self.table_blocks)
         return out
 
     def status(self) -> int:

@@ -10,6 +10,13 @@ static thread_local int g_last_launches = 0;
 static inline bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
 constexpr int32_t kMaxBlocksArg = INT32_MAX / kPageTokens;      // 16 * max_blocks must fit an int
 
+// A NULL block table means a contiguous cache: unit (b, h) owns pages [u * max_blocks, (u + 1) * max_blocks),
+// u = b * n_kv_heads + h.  The pool must hold them all.
+static inline bool contiguous_pool_too_small(const spark_params* p, const void* block_table, int32_t max_blocks)
+{
+    return !block_table && static_cast<int64_t>(p->batch) * p->n_kv_heads * max_blocks > p->n_pool_pages;
+}
+
 spark_status spark::check_params(const spark_params* p)
 {
     if (!p) return SPARK_ERR_NULL;
@@ -88,11 +95,12 @@ spark_status spark_compress(const spark_params* p, const void* q_win, const void
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!q_win || !k || !v || !seq_lens || !pages || !block_table || !qnorm || !packed_lens || !workspace)
+    if (!q_win || !k || !v || !seq_lens || !pages || !qnorm || !packed_lens || !workspace)
         return SPARK_ERR_NULL;
     if (p->window < 1 || max_seq_tokens < 0 || max_blocks < 0 || max_blocks > kMaxBlocksArg) return SPARK_ERR_BAD_SHAPE;
     if (stride_t < p->head_dim || stride_b < 0 || stride_h < 0) return SPARK_ERR_BAD_SHAPE;
     if (misaligned(pages, 16) || misaligned(qnorm, 16)) return SPARK_ERR_BAD_SHAPE;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
     // vector loads of K/V rows need 16-byte aligned rows
     const int e = (p->dtype == SPARK_BF16) ? 2 : 4;
     if ((reinterpret_cast<uintptr_t>(k) & 15) || (reinterpret_cast<uintptr_t>(v) & 15) ||
@@ -123,8 +131,9 @@ spark_status spark_append(const spark_params* p, const void* k_new, const void* 
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!k_new || !v_new || !pages || !block_table || !qnorm || !packed_lens || !workspace) return SPARK_ERR_NULL;
+    if (!k_new || !v_new || !pages || !qnorm || !packed_lens || !workspace) return SPARK_ERR_NULL;
     if (max_blocks < 1 || max_blocks > kMaxBlocksArg) return SPARK_ERR_BAD_SHAPE;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
     if (misaligned(pages, 16) || misaligned(k_new, 16) || misaligned(v_new, 16) || misaligned(qnorm, 16))
         return SPARK_ERR_BAD_SHAPE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < kWorkspaceHeader) return SPARK_ERR_WORKSPACE;
@@ -142,8 +151,9 @@ spark_status spark_decode_attn(const spark_params* p, const void* q, const void*
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!q || !pages || !block_table || !packed_lens || !qnorm || !out || !workspace) return SPARK_ERR_NULL;
+    if (!q || !pages || !packed_lens || !qnorm || !out || !workspace) return SPARK_ERR_NULL;
     if (max_blocks < 0 || max_blocks > kMaxBlocksArg) return SPARK_ERR_BAD_SHAPE;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
     // the kernels read q and qnorm and write out with 16-byte vector accesses
     if (misaligned(pages, 16) || misaligned(q, 16) || misaligned(qnorm, 16) || misaligned(out, 16) ||
         misaligned(lse, 4))
@@ -163,7 +173,8 @@ spark_status spark_unpack_pages(const spark_params* p, const void* pages, const 
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!pages || !block_table || !packed_lens) return SPARK_ERR_NULL;
+    if (!pages || !packed_lens) return SPARK_ERR_NULL;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
     if (max_tokens < 0 || max_blocks < 0 || max_blocks > kMaxBlocksArg) return SPARK_ERR_BAD_SHAPE;
     if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
         return SPARK_ERR_BAD_SHAPE;
@@ -177,7 +188,8 @@ spark_status spark_unpack_value_masks(const spark_params* p, const void* pages, 
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!pages || !block_table || !packed_lens || !vmask) return SPARK_ERR_NULL;
+    if (!pages || !packed_lens || !vmask) return SPARK_ERR_NULL;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
     if (max_tokens < 0 || max_blocks < 0) return SPARK_ERR_BAD_SHAPE;
     if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
         return SPARK_ERR_BAD_SHAPE;

@@ -250,12 +250,13 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     }
     __syncthreads();
 
-    const int page_id = A.block_table[(static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk];
+    const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+    const int64_t page_id = A.block_table ? A.block_table[entry] : entry;     // no table: contiguous cache
     if (page_id < 0 || page_id >= A.n_pool_pages) {
         if (threadIdx.x == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
         return;
     }
-    uint4* dst = reinterpret_cast<uint4*>(A.pages + static_cast<int64_t>(page_id) * L.page_bytes);
+    uint4* dst = reinterpret_cast<uint4*>(A.pages + page_id * L.page_bytes);
     for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
         dst[i] = reinterpret_cast<const uint4*>(image)[i];
 }
@@ -292,12 +293,13 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
         if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
         return;
     }
-    const int page_id = A.block_table[(static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk];
+    const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+    const int64_t page_id = A.block_table ? A.block_table[entry] : entry;
     if (page_id < 0 || page_id >= A.n_pool_pages) {
         if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
         return;
     }
-    unsigned char* page = A.pages + static_cast<int64_t>(page_id) * L.page_bytes;
+    unsigned char* page = A.pages + page_id * L.page_bytes;
     if (p == 0) {                                             // first token of a page: clear it
         for (int i = lane; i < L.page_bytes / 16; i += 32) reinterpret_cast<uint4*>(page)[i] = make_uint4(0, 0, 0, 0);
         __syncwarp();
@@ -363,8 +365,8 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
     const int64_t unit = static_cast<int64_t>(b) * A.Hkv + h;
     const unsigned char* page = nullptr;
     if (blk * kPageTokens < len) {
-        const int id = A.block_table[unit * A.max_blocks + blk];
-        if (id >= 0 && id < A.n_pool_pages) page = A.pages + static_cast<int64_t>(id) * L.page_bytes;
+        const int64_t id = A.block_table ? A.block_table[unit * A.max_blocks + blk] : unit * A.max_blocks + blk;
+        if (id >= 0 && id < A.n_pool_pages) page = A.pages + id * L.page_bytes;
     }
     const int t0 = blk * kPageTokens;
     const int64_t row0 = unit * A.max_tokens + t0;

@@ -46,16 +46,19 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
     const int NS = A.nslots;
     const int max_tokens = A.max_blocks * kPageTokens;
 
-    decode_prologue(A, C, tid);
+    prefetch_block_table(A, tid, kDecodeThreads);
+    if (tid == 0) pdl_launch_dependents();
+    if (warp == kConsumerWarps) {
+        producer_prologue(A, C, lane, kDecodeThreads);
+        int p0, p1;
+        cta_range(*C.plan, static_cast<int>(blockIdx.x), p0, p1);
+        producer_loop(A, C, ring, p0, p1, lane);
+        return;
+    }
+    consumer_wait_plan(kDecodeThreads);
     const int* prefix = C.prefix;
     int c0, c1;
     cta_range(*C.plan, static_cast<int>(blockIdx.x), c0, c1);
-
-    if (tid == 0) pdl_launch_dependents();
-    if (warp == kConsumerWarps) {
-        producer_loop(A, C, ring, c0, c1, lane);
-        return;
-    }
     pdl_dependency_wait();                                 // q, qnorm, out and the workspace from here on
     write_empty_sequences<kConsumerThreads>(A, prefix, tid);
 
@@ -227,6 +230,23 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+bool device_info(int* dev, DeviceInfo* info)
+{
+    static DeviceInfo table[kMaxDevices];
+    static unsigned char known[kMaxDevices] = {};
+    if (cudaGetDevice(dev) != cudaSuccess || *dev < 0 || *dev >= kMaxDevices) return false;
+    if (!known[*dev]) {                                   // a racing first call writes the same values
+        DeviceInfo d;
+        if (cudaDeviceGetAttribute(&d.n_sms, cudaDevAttrMultiProcessorCount, *dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, *dev) != cudaSuccess)
+            return false;
+        table[*dev] = d;
+        known[*dev] = 1;
+    }
+    *info = table[*dev];
+    return true;
+}
+
 size_t decode_workspace_bytes(const spark_params& p)
 {
     const int G = p.n_q_heads / p.n_kv_heads;
@@ -238,8 +258,10 @@ size_t decode_workspace_bytes(const spark_params& p)
 }
 
 template <int G>
-static spark_status launch_f32(const DecodeArgs& A0, int n_sms, int smem_optin, cudaStream_t stream)
+static spark_status launch_f32(const DecodeArgs& A0, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
+    static unsigned char smem_raised[kMaxDevices] = {};
+    const int n_sms = info.n_sms, smem_optin = info.smem_optin;
     DecodeArgs A = A0;
     using S = SmemF32<G>;
     A.pps = 2;
@@ -249,25 +271,23 @@ static spark_status launch_f32(const DecodeArgs& A0, int n_sms, int smem_optin, 
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
     const size_t smem = S::kRing + static_cast<size_t>(ns) * A.slot_stride;
-    if (cudaFuncSetAttribute(decode_f32_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem)) != cudaSuccess)
-        return SPARK_ERR_CUDA;
+    if (!allow_max_smem(decode_f32_kernel<G>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
     return launch_decode_kernel(decode_f32_kernel<G>, grid, kDecodeThreads, smem, stream, A) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
-spark_status launch_decode_f32(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream)
+spark_status launch_decode_f32(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
     switch (G) {
-        case 1: return launch_f32<1>(A, n_sms, smem_optin, stream);
-        case 2: return launch_f32<2>(A, n_sms, smem_optin, stream);
-        case 3: return launch_f32<3>(A, n_sms, smem_optin, stream);
-        case 4: return launch_f32<4>(A, n_sms, smem_optin, stream);
-        case 5: return launch_f32<5>(A, n_sms, smem_optin, stream);
-        case 6: return launch_f32<6>(A, n_sms, smem_optin, stream);
-        case 7: return launch_f32<7>(A, n_sms, smem_optin, stream);
-        case 8: return launch_f32<8>(A, n_sms, smem_optin, stream);
+        case 1: return launch_f32<1>(A, dev, info, stream);
+        case 2: return launch_f32<2>(A, dev, info, stream);
+        case 3: return launch_f32<3>(A, dev, info, stream);
+        case 4: return launch_f32<4>(A, dev, info, stream);
+        case 5: return launch_f32<5>(A, dev, info, stream);
+        case 6: return launch_f32<6>(A, dev, info, stream);
+        case 7: return launch_f32<7>(A, dev, info, stream);
+        case 8: return launch_f32<8>(A, dev, info, stream);
         default: return SPARK_ERR_UNSUPPORTED;
     }
 }
@@ -278,11 +298,9 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
                            size_t workspace_bytes, cudaStream_t stream, int* launches)
 {
     (void)workspace_bytes;
-    int dev = 0, n_sms = 0, smem_optin = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-        return SPARK_ERR_CUDA;
+    int dev = 0;
+    DeviceInfo info;
+    if (!device_info(&dev, &info)) return SPARK_ERR_CUDA;
     const int G = p.n_q_heads / p.n_kv_heads;
     const size_t units = static_cast<size_t>(p.batch) * p.n_kv_heads;
     DecodeArgs A;
@@ -298,8 +316,8 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.partials = reinterpret_cast<float*>(ws + kWorkspaceHeader + align_up(units * sizeof(int), 256));
     A.nslots = 0; A.slot_stride = 0; A.pps = 1;
     A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
-    const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, n_sms, smem_optin, stream)
-                                                    : launch_decode_f32(G, A, n_sms, smem_optin, stream);
+    const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, dev, info, stream)
+                                                    : launch_decode_f32(G, A, dev, info, stream);
     if (st == SPARK_OK) ++*launches;
     return st;
 }

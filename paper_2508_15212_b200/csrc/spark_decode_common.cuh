@@ -15,7 +15,8 @@
 namespace spark {
 
 constexpr int kMaxSlots = 32;
-constexpr unsigned kSpinLimit = 1u << 20;    // bounded mbarrier waits
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // every device-side wait gives up after one second
+constexpr unsigned kClockEvery = 256;                        // polls between two looks at the clock
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kRec = kHeadDim + 4;           // floats per head record: 128 outputs, running max, running sum, pad
 constexpr float kLn2 = 0.6931471805599453f;
@@ -46,12 +47,16 @@ struct DecodeArgs {
 constexpr int kCtrlBytes = 1024;                                 // full[32], empty[32], flags, plan
 constexpr int kPrefixBytes = ((kMaxBatch + 1) * 4 + 15) / 16 * 16;
 
-// Bytes of the shared merge area for `nw` consumer warps and `g` heads.  The final combine reuses it
-// for the (m, l) pairs of up to kMaxCtas parts followed by one float4 per consumer thread.
+// Shared merge area for `nw` consumer warps and `g` heads: the warps' states ([warp][head][kRec] floats),
+// reused by the final combine for the weights of up to kMaxCtas parts, the heads' (M, L) and one float4
+// per consumer thread; behind it the weights of the warps ([head][32]) and the heads' (M, L).
+__host__ __device__ constexpr int merge_state_floats(int nw, int g)
+{
+    return nw * g * kRec > kMaxCtas * g * 2 + nw * 32 * 4 ? nw * g * kRec : kMaxCtas * g * 2 + nw * 32 * 4;
+}
 __host__ __device__ constexpr int merge_bytes(int nw, int g)
 {
-    return nw * g * kRec * 4 > kMaxCtas * g * 8 + nw * 32 * 16 ? nw * g * kRec * 4
-                                                               : kMaxCtas * g * 8 + nw * 32 * 16;
+    return (merge_state_floats(nw, g) + g * 32 + g * 2 + 2) * 4;
 }
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
@@ -84,12 +89,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
         : "memory");
     return ok != 0;
 }
-// Wait with an iteration limit.  On expiry (or if another thread already gave up) the CTA-wide abort
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Expiry test of a polling loop: looks at the nanosecond clock every kClockEvery polls (the first look
+// only records the start), so a wait is bounded by wall time, not by how fast the poll happens to spin.
+struct WaitClock {
+    unsigned it = 0;
+    unsigned long long t0 = 0;
+    __device__ __forceinline__ bool expired()
+    {
+        if ((++it & (kClockEvery - 1)) != 0) return false;
+        const unsigned long long now = global_ns();
+        if (t0 == 0) { t0 = now; return false; }
+        return now - t0 > kWaitLimitNs;
+    }
+};
+// Wait with a time limit.  On expiry (or if another thread already gave up) the CTA-wide abort
 // flag is set, the status word records the timeout and the caller carries on without the data; the
 // kernel then finishes structurally (same barriers) and returns.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volatile int* abort_flag, int* status)
 {
-    for (unsigned it = 0; it < kSpinLimit; ++it) {
+    WaitClock wc;
+    while (!wc.expired()) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -119,9 +144,9 @@ __device__ __forceinline__ uint64_t policy_evict_first()
 __device__ __forceinline__ bool slot_wait(uint64_t* full, volatile int* seq, int slot, int round,
                                           volatile int* abort_flag, int* status)
 {
-    unsigned it = 0;
+    WaitClock wc;
     while (seq[slot] != round + 1) {
-        if (++it >= kSpinLimit || *abort_flag) {
+        if (wc.expired() || *abort_flag) {
             if (!*abort_flag) { *abort_flag = 1; record_error(status, SPARK_ERR_DEVICE_TIMEOUT); }
             return false;
         }
@@ -233,70 +258,95 @@ __device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
     return c;
 }
 
-// Barrier init (one thread of warp 1), the steps-per-sequence prefix and the plan (warp 0).
-// Ends with __syncthreads().
-__device__ __forceinline__ void decode_prologue(const DecodeArgs& A, const Ctrl& C, int tid)
+// Start of the kernel.  The PRODUCER warp alone reads packed_lens, builds the steps-per-sequence prefix and
+// the plan, initialises the ring barriers, and then arrives (without waiting) on hardware barrier 2; it
+// goes straight on to its first page copies.  The consumer warps wait on barrier 2 for the plan.  So the
+// chain from launch to the first bytes in flight is: packed_lens (one global round trip) -> plan -> page
+// ids -> bulk copies, with no CTA-wide barrier in between.
+//
+// All threads first ask the L2 to fetch the block table (when there is one): the producer's page-id
+// loads then find their lines on the way instead of starting a second cold DRAM round trip behind
+// packed_lens.
+constexpr int kPlanBarrier = 2;
+constexpr int64_t kTablePrefetchMax = 8 << 20;             // bytes of block table asked for at most
+
+__device__ __forceinline__ void prefetch_block_table(const DecodeArgs& A, int tid, int n_threads)
 {
-    const int warp = tid >> 5, lane = tid & 31;
+    if (!A.block_table) return;
+    int64_t bytes = static_cast<int64_t>(A.B) * A.Hkv * A.max_blocks * 4;
+    if (bytes > kTablePrefetchMax) bytes = kTablePrefetchMax;
+    const char* base = reinterpret_cast<const char*>(A.block_table);
+    for (int64_t o = (static_cast<int64_t>(blockIdx.x) * n_threads + tid) * 128; o < bytes;
+         o += static_cast<int64_t>(gridDim.x) * n_threads * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + o));
+}
+
+__device__ __forceinline__ void producer_prologue(const DecodeArgs& A, const Ctrl& C, int lane, int n_threads)
+{
     const int max_tokens = A.max_blocks * kPageTokens;
-    if (warp == 1) C.seq[lane] = 0;
-    if (tid == 32) {
-        for (int s = 0; s < A.nslots; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], 1); }
-        *C.abort_flag = 0;
-        *C.last_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 0) {
-        int running = 0, smin = 0x7fffffff, smax = 0;
-        for (int b0 = 0; b0 < A.B; b0 += 32) {
-            const int b = b0 + lane;
-            int st = 0;
-            if (b < A.B) {
-                const int len = A.lens[b];
-                if (len < 0 || len > max_tokens) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
-                st = steps_of(clamp_len(len, max_tokens), A.pps);
-                smin = min(smin, st);
-                smax = max(smax, st);
-            }
-            int inc = st;
+    // packed_lens first: everything else of the prologue fits under this load's latency
+    int first_len = 0;
+    if (lane < A.B) first_len = A.lens[lane];
+    if (lane < A.nslots) { mbar_init(&C.full[lane], 1); mbar_init(&C.empty[lane], 1); }
+    C.seq[lane] = 0;
+    if (lane == 0) { *C.abort_flag = 0; *C.last_flag = 0; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    int running = 0, smin = 0x7fffffff, smax = 0;
+    for (int b0 = 0; b0 < A.B; b0 += 32) {
+        const int b = b0 + lane;
+        int st = 0;
+        if (b < A.B) {
+            const int len = b0 == 0 ? first_len : A.lens[b];
+            if (len < 0 || len > max_tokens) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+            st = steps_of(clamp_len(len, max_tokens), A.pps);
+            smin = min(smin, st);
+            smax = max(smax, st);
+        }
+        int inc = st;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int n = __shfl_up_sync(kFull, inc, o);
-                if (lane >= o) inc += n;
-            }
-            if (b < A.B) C.prefix[b + 1] = running + inc;
-            running += __shfl_sync(kFull, inc, 31);
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(kFull, inc, o);
+            if (lane >= o) inc += n;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            smin = min(smin, __shfl_xor_sync(kFull, smin, o));
-            smax = max(smax, __shfl_xor_sync(kFull, smax, o));
-        }
-        if (lane == 0) {
-            C.prefix[0] = 0;
-            Plan pl;
-            const int nct = static_cast<int>(gridDim.x), units = A.B * A.Hkv;
-            pl.total = A.Hkv * running;
-            pl.chunk = (pl.total + nct - 1) / nct;
-            pl.aligned = 0; pl.unit_steps = smax; pl.q = 0; pl.rem = 0;
-            if (smin == smax && smax > 0 && units <= nct) {
-                const int q = nct / units;
-                const int makespan = (smax + q - 1) / q;
-                if (q >= 2 && makespan * 25 <= pl.chunk * 26) {          // within 4 % of the even split
-                    pl.aligned = 1; pl.q = q; pl.rem = nct - q * units;
-                }
-            } else if (smin == smax && smax > 0) {
-                const int q = units / nct, rem = units - q * nct;
-                const int makespan = (q + (rem ? 1 : 0)) * smax;
-                if (makespan * 4 <= pl.chunk * 5) {                      // within 25 % of the even split
-                    pl.aligned = 2; pl.q = q; pl.rem = rem;
-                }
-            }
-            *C.plan = pl;
-        }
+        if (b < A.B) C.prefix[b + 1] = running + inc;
+        running += __shfl_sync(kFull, inc, 31);
     }
-    __syncthreads();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        smin = min(smin, __shfl_xor_sync(kFull, smin, o));
+        smax = max(smax, __shfl_xor_sync(kFull, smax, o));
+    }
+    if (lane == 0) {
+        C.prefix[0] = 0;
+        Plan pl;
+        const int nct = static_cast<int>(gridDim.x), units = A.B * A.Hkv;
+        pl.total = A.Hkv * running;
+        pl.chunk = (pl.total + nct - 1) / nct;
+        pl.aligned = 0; pl.unit_steps = smax; pl.q = 0; pl.rem = 0;
+        if (smin == smax && smax > 0 && units <= nct) {
+            const int q = nct / units;
+            const int makespan = (smax + q - 1) / q;
+            if (q >= 2 && makespan * 25 <= pl.chunk * 26) {          // within 4 % of the even split
+                pl.aligned = 1; pl.q = q; pl.rem = nct - q * units;
+            }
+        } else if (smin == smax && smax > 0) {
+            const int q = units / nct, rem = units - q * nct;
+            const int makespan = (q + (rem ? 1 : 0)) * smax;
+            if (makespan * 4 <= pl.chunk * 5) {                      // within 25 % of the even split
+                pl.aligned = 2; pl.q = q; pl.rem = rem;
+            }
+        }
+        *C.plan = pl;
+    }
+    __syncwarp();
+    asm volatile("bar.arrive %0, %1;" ::"n"(kPlanBarrier), "r"(n_threads) : "memory");
+}
+
+// consumer side of the prologue: returns once the plan, the prefix and the ring barriers are in place
+__device__ __forceinline__ void consumer_wait_plan(int n_threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(kPlanBarrier), "r"(n_threads) : "memory");
 }
 
 // This CTA's run of steps [c0, c1) on the line.
@@ -355,12 +405,13 @@ __device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctr
     id0 = -1; id1 = -1;
     if (!active) return;
     const Segment s = locate(C.prefix, A.B, A.Hkv, g, c1);
-    const int32_t* bt = A.block_table + (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
-    id0 = bt[A.pps * s.i0];
+    const int64_t row = (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
+    const int32_t* bt = A.block_table ? A.block_table + row : nullptr;       // no table: pages of a unit are consecutive
+    id0 = bt ? bt[A.pps * s.i0] : static_cast<int>(row + A.pps * s.i0);
     if (A.pps == 2) {                                       // second page of the step, if the sequence has one
         const int len = clamp_len(A.lens[s.b], A.max_blocks * kPageTokens);
         if (2 * s.i0 + 1 < (len + kPageTokens - 1) / kPageTokens) {
-            id1 = bt[2 * s.i0 + 1];
+            id1 = bt ? bt[2 * s.i0 + 1] : static_cast<int>(row + 2 * s.i0 + 1);
             if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
         }
     }
@@ -389,7 +440,7 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
         // (hidden behind the wait for free slots) except in the first revolution, where every slot is
         // free and the copies go out first
         if (round > 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
-        unsigned it = 0;
+        WaitClock wc;
         while (__any_sync(kFull, pending)) {
             if (pending && (round == 0 || mbar_try_wait(empty, (round - 1) & 1))) {
                 const unsigned bytes = L.page_bytes * (cur1 >= 0 ? 2u : 1u);
@@ -402,16 +453,18 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
                 last_round = round;
                 pending = false;
             }
-            if (++it >= kSpinLimit || *C.abort_flag) { live = false; break; }
+            if (wc.expired() || *C.abort_flag) { live = false; break; }
         }
         if (!live) break;
         if (round == 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
     }
     if (!live) {
         if (lane == 0) { *C.abort_flag = 1; record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT); }
-        if (last_round >= 0)                               // let this lane's copy in flight land
-            for (unsigned it = 0; it < kSpinLimit; ++it)
+        if (last_round >= 0) {                             // let this lane's copy in flight land
+            WaitClock wc;
+            while (!wc.expired())
                 if (mbar_try_wait(full, last_round & 1)) break;
+        }
     }
 }
 
@@ -433,36 +486,62 @@ __device__ __forceinline__ void write_empty_sequences(const DecodeArgs& A, const
 // ([warp][G][kRec]: 128 unnormalised outputs, m, l) and publish the unit's result: directly when this
 // CTA covers the whole unit, else as a partial followed by the last-arriver merge.  Called by all
 // consumer threads after a consumer_sync(); ends with a consumer_sync().
+//
+// Both merges are laid out so that no thread walks a chain of dependent shared-memory loads: the
+// log-sum-exp weights of the parts are computed once, by one warp per head with warp reductions, and the
+// weighted sums then read independent operands.
 template <int G, int NW>
 __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctrl& C, float* merge,
                                                   const Segment& sg, int tid)
 {
     constexpr int NT = NW * 32;
+    static_assert(G <= NW && NW <= 32, "one warp per head computes the weights of up to 32 warps");
     const int b = sg.b, h = sg.h;
+    const int warp = tid >> 5, lane = tid & 31;
     int first_cta, n_parts;
     unit_parts(*C.plan, sg.unit_start, sg.steps_b, first_cta, n_parts);
     const int unit = b * A.Hkv + h;
-    float* part_out = A.partials + static_cast<int64_t>(blockIdx.x + unit) * G * kRec;
-    for (int idx = tid; idx < G * kHeadDim; idx += NT) {
-        const int gg = idx / kHeadDim, c = idx - gg * kHeadDim;
-        float M = -INFINITY;
+    float* wts = merge + merge_state_floats(NW, G);           // [G][32] weights of the warps, then [G][2] (M, L)
+    float* ML = wts + G * 32;
+    // ---- weights of the warps: warp g serves head g, lane w holds warp w's (m, l) ----
+    if (warp < G) {
+        const float m = lane < NW ? merge[(lane * G + warp) * kRec + kHeadDim] : -INFINITY;
+        const float l = lane < NW ? merge[(lane * G + warp) * kRec + kHeadDim + 1] : 0.f;
+        float M = m;
 #pragma unroll
-        for (int w = 0; w < NW; ++w) M = fmaxf(M, merge[(w * G + gg) * kRec + kHeadDim]);
-        float Ls = 0.f, O = 0.f;
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+        const float wt = (m == -INFINITY) ? 0.f : exp2f(m - M);
+        float Ls = l * wt;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(kFull, Ls, o);
+        wts[warp * 32 + lane] = wt;
+        if (lane == 0) { ML[2 * warp] = M; ML[2 * warp + 1] = Ls; }
+    }
+    consumer_sync<NT>();
+    // ---- weighted sums: a thread owns two channels of one head ----
+    float* part_out = A.partials + static_cast<int64_t>(blockIdx.x + unit) * G * kRec;
+    for (int idx = tid; idx < G * (kHeadDim / 2); idx += NT) {
+        const int gg = idx / (kHeadDim / 2), c2 = idx - gg * (kHeadDim / 2);
+        float2 v[NW];
+#pragma unroll
+        for (int w = 0; w < NW; ++w) v[w] = *reinterpret_cast<const float2*>(merge + (w * G + gg) * kRec + 2 * c2);
+        float2 O = make_float2(0.f, 0.f);
 #pragma unroll
         for (int w = 0; w < NW; ++w) {
-            const float* r = merge + (w * G + gg) * kRec;
-            const float f = exp2f(r[kHeadDim] - M);
-            Ls = fmaf(r[kHeadDim + 1], f, Ls);
-            O = fmaf(r[c], f, O);
+            const float f = wts[gg * 32 + w];
+            O.x = fmaf(v[w].x, f, O.x);
+            O.y = fmaf(v[w].y, f, O.y);
         }
+        const float M = ML[2 * gg], Ls = ML[2 * gg + 1];
         if (n_parts == 1) {
-            A.out[(static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + c] = O / Ls;
-            if (c == 0 && A.lse)
+            const float inv = 1.0f / Ls;
+            *reinterpret_cast<float2*>(A.out + (static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + 2 * c2) =
+                make_float2(O.x * inv, O.y * inv);
+            if (c2 == 0 && A.lse)
                 A.lse[static_cast<int64_t>(b) * A.Hq + h * G + gg] = (M + log2f(Ls)) * kLn2;
         } else {
-            part_out[gg * kRec + c] = O;
-            if (c == 0) { part_out[gg * kRec + kHeadDim] = M; part_out[gg * kRec + kHeadDim + 1] = Ls; }
+            *reinterpret_cast<float2*>(part_out + gg * kRec + 2 * c2) = O;
+            if (c2 == 0) *reinterpret_cast<float2*>(part_out + gg * kRec + kHeadDim) = make_float2(M, Ls);
         }
     }
     if (n_parts > 1) {
@@ -478,20 +557,22 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
         consumer_sync<NT>();
         if (*C.last_flag) {
             // Last CTA of this unit: merge all partials.  Every load is issued before the first use:
-            // thread (ph, g, c4) fetches channels 4*c4..4*c4+3 of head g for parts ph, ph+PH, ...
-            // while the (m, l) pairs of all parts go to shared memory; after one barrier the weights
-            // are known, and the weighted sums are reduced over ph through shared memory.
+            // thread (ph, g, c4) fetches channels 4*c4..4*c4+3 of head g for parts ph, ph+PH, ...;
+            // meanwhile warp g turns the (m, l) pairs of head g into weights (lane = part) and the
+            // head's (M, L).  After one barrier the weights are known, and the weighted sums are
+            // reduced over ph through shared memory.
             constexpr int TPG = G * 32;                  // threads per part group
             constexpr int PH = NT / TPG;                 // part groups
-            constexpr int kBatch = 16;
+            constexpr int kBatch = 8;
+            constexpr int kMlRegs = kMaxCtas / 32;       // (m, l) pairs a lane may hold
             constexpr int64_t kStride = static_cast<int64_t>(G) * kRec;
-            float* ml = merge;                           // [n_parts][G][2], n_parts <= kMaxCtas
+            float* pw = merge;                           // [n_parts][G] weights, n_parts <= kMaxCtas
+            float* pML = merge + kMaxCtas * G;           // [G][2]
             float4* red = reinterpret_cast<float4*>(merge + kMaxCtas * G * 2);
             const float* base = A.partials + static_cast<int64_t>(first_cta + unit) * G * kRec;
             const int ph = tid / TPG, rem = tid - ph * TPG, gg = rem >> 5, c4 = rem & 31;
             const bool worker = ph < PH;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            float M = -INFINITY;
             for (int p0 = 0; p0 < n_parts; p0 += kBatch * PH) {
                 float4 o4[kBatch];
 #pragma unroll
@@ -502,30 +583,43 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 if (p0 == 0) {
-                    for (int i = tid; i < n_parts * G; i += NT) {
-                        const int p = i / G, g2 = i - p * G;
-                        const float2 v = *reinterpret_cast<const float2*>(base + p * kStride + g2 * kRec + kHeadDim);
-                        ml[2 * i] = v.x;
-                        ml[2 * i + 1] = v.y;
+                    if (warp < G) {
+                        float2 ml[kMlRegs];
+#pragma unroll
+                        for (int k = 0; k < kMlRegs; ++k) {
+                            const int p = k * 32 + lane;
+                            ml[k] = p < n_parts ? *reinterpret_cast<const float2*>(base + p * kStride + warp * kRec + kHeadDim)
+                                                : make_float2(-INFINITY, 0.f);
+                        }
+                        float M = -INFINITY;
+#pragma unroll
+                        for (int k = 0; k < kMlRegs; ++k) M = fmaxf(M, ml[k].x);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+                        float Ls = 0.f;
+#pragma unroll
+                        for (int k = 0; k < kMlRegs; ++k) {
+                            const int p = k * 32 + lane;
+                            const float wt = (ml[k].x == -INFINITY) ? 0.f : exp2f(ml[k].x - M);
+                            Ls = fmaf(ml[k].y, wt, Ls);
+                            if (p < n_parts) pw[p * G + warp] = wt;
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(kFull, Ls, o);
+                        if (lane == 0) { pML[2 * warp] = M; pML[2 * warp + 1] = Ls; }
                     }
                     consumer_sync<NT>();
-                    if (worker)
-                        for (int p = 0; p < n_parts; ++p) M = fmaxf(M, ml[2 * (p * G + gg)]);
                 }
 #pragma unroll
                 for (int k = 0; k < kBatch; ++k) {
                     const int p = p0 + k * PH + ph;
                     if (worker && p < n_parts) {
-                        const float f = exp2f(ml[2 * (p * G + gg)] - M);
+                        const float f = pw[p * G + gg];
                         acc.x = fmaf(o4[k].x, f, acc.x); acc.y = fmaf(o4[k].y, f, acc.y);
                         acc.z = fmaf(o4[k].z, f, acc.z); acc.w = fmaf(o4[k].w, f, acc.w);
                     }
                 }
             }
-            float Ls = 0.f;
-            if (worker)
-                for (int p = 0; p < n_parts; ++p)
-                    Ls = fmaf(ml[2 * (p * G + gg) + 1], exp2f(ml[2 * (p * G + gg)] - M), Ls);
             if (PH > 1) {
                 if (worker && ph > 0) red[tid] = acc;
                 consumer_sync<NT>();
@@ -537,6 +631,7 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
                     }
             }
             if (ph == 0) {
+                const float M = pML[2 * gg], Ls = pML[2 * gg + 1];
                 const float inv = 1.0f / Ls;
                 *reinterpret_cast<float4*>(A.out + (static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + 4 * c4) =
                     make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -551,8 +646,24 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Device properties the launchers need, looked up once per device and then served from a table
+// (spark_decode.cu); `dev` is the current device.
+struct DeviceInfo { int n_sms; int smem_optin; };
+bool device_info(int* dev, DeviceInfo* info);
+
+// Raises a kernel's dynamic shared-memory limit to the device maximum, once per device and kernel.
+constexpr int kMaxDevices = 64;
+template <typename Kernel> inline bool allow_max_smem(Kernel kernel, int dev, int smem_optin, unsigned char (&done)[kMaxDevices])
+{
+    if (dev < 0 || dev >= kMaxDevices) return false;
+    if (done[dev]) return true;                           // a racing first call only repeats the same setting
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin) != cudaSuccess) return false;
+    done[dev] = 1;
+    return true;
+}
+
 // per-dtype launchers (spark_decode.cu: fp32 storage, spark_decode_mma.cu: bf16 storage)
-spark_status launch_decode_f32(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream);
-spark_status launch_decode_bf16(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream);
+spark_status launch_decode_f32(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream);
+spark_status launch_decode_bf16(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream);
 
 }  // namespace spark

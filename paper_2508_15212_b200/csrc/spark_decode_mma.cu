@@ -207,25 +207,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
     const int NS = A.nslots;
     const int max_tokens = A.max_blocks * kPageTokens;
 
-    decode_prologue(A, C, tid);
+    prefetch_block_table(A, tid, kThreads);
+    if (tid == 0) pdl_launch_dependents();
+    if (warp == kNW) {
+        producer_prologue(A, C, lane, kThreads);
+        int p0, p1;
+        cta_range(*C.plan, static_cast<int>(blockIdx.x), p0, p1);
+        producer_loop(A, C, ring, p0, p1, lane);
+        return;
+    }
+    consumer_wait_plan(kThreads);
     const int* prefix = C.prefix;
     int c0, c1;
     cta_range(*C.plan, static_cast<int>(blockIdx.x), c0, c1);
-
-#ifdef SPARK_CTA_TIMING
-    unsigned long long t_start = 0, t_first = 0, t_probe[12];
-    int n_probe = 0;
-    for (int i = 0; i < 12; ++i) t_probe[i] = 0;
-#define SPARK_PROBE() do { if (tid == 0 && n_probe < 12) { asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_probe[n_probe])); ++n_probe; } } while (0)
-    if (tid == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_start));
-#else
-#define SPARK_PROBE() do { } while (0)
-#endif
-    if (tid == 0) pdl_launch_dependents();
-    if (warp == kNW) {
-        producer_loop(A, C, ring, c0, c1, lane);
-        return;
-    }
     pdl_dependency_wait();                                 // q, qnorm, out and the workspace from here on
     write_empty_sequences<kNT>(A, prefix, tid);
 
@@ -293,7 +287,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
             hv[e] = (2 * c + e < G) && (!kShared8 || c < 2);
             qsum[e] = hv[e] ? qsum_s[2 * c + e] : 0.f;
         }
-        SPARK_PROBE();      // setup done
 
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
         float thr[2] = {hv[0] ? -INFINITY : INFINITY, hv[1] ? -INFINITY : INFINITY};
@@ -309,9 +302,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
             const bool ok = slot_wait(C.full, C.seq, slot, round, C.abort_flag, A.status);
             const unsigned page = ring_u + static_cast<unsigned>(slot) * A.slot_stride;
             const int n_valid = min(kPageTokens, len - i * kPageTokens);
-#ifdef SPARK_CTA_TIMING
-            if (tid == 0 && t_first == 0) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_first));
-#endif
             if (ok) {
                 // ---------------- scores of the page's 16 tokens (rows r and r+8) ----------------
                 float d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f}, d3[4] = {0.f, 0.f, 0.f, 0.f};
@@ -452,7 +442,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
             __syncwarp();
             if (lane == 0) mbar_arrive(&C.empty[slot]);
         }
-        SPARK_PROBE();      // steps done (warp 0)
 
         // ---------------- hand the warp state to the merge ----------------
         {
@@ -481,29 +470,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                 }
         }
         consumer_sync<kNT>();
-        SPARK_PROBE();      // all warps done
         merge_and_publish<G, kNW>(A, C, merge, sg, tid);
-        SPARK_PROBE();      // published
         g += sg.n;
         base += sg.n;
     }
-#ifdef SPARK_CTA_TIMING
-    if (tid == 0) {
-        unsigned long long t_end;
-        unsigned smid;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_end));
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        unsigned long long* rec = reinterpret_cast<unsigned long long*>(
-            A.partials + static_cast<int64_t>(kMaxCtas + A.B * A.Hkv - 1 - blockIdx.x) * G * kRec);
-        rec[0] = t_start; rec[1] = t_first; rec[2] = t_end; rec[3] = smid;
-        for (int i = 0; i < 12; ++i) rec[4 + i] = t_probe[i];
-    }
-#endif
 }
 
 template <int G, bool kPV>
-static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin, cudaStream_t stream)
+static spark_status launch_bf16(const DecodeArgs& A0, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
+    static unsigned char smem_raised[kMaxDevices] = {};
+    const int n_sms = info.n_sms, smem_optin = info.smem_optin;
     DecodeArgs A = A0;
     using S = SmemBf16<G, kPV>;
     A.pps = 1;
@@ -513,26 +490,24 @@ static spark_status launch_bf16(const DecodeArgs& A0, int n_sms, int smem_optin,
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
     const size_t smem = S::kRing + static_cast<size_t>(ns) * A.slot_stride;
-    if (cudaFuncSetAttribute(decode_bf16_kernel<G, kPV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem)) != cudaSuccess)
-        return SPARK_ERR_CUDA;
+    if (!allow_max_smem(decode_bf16_kernel<G, kPV>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
     return launch_decode_kernel(decode_bf16_kernel<G, kPV>, grid, kThreads, smem, stream, A) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
-spark_status launch_decode_bf16(int G, const DecodeArgs& A, int n_sms, int smem_optin, cudaStream_t stream)
+spark_status launch_decode_bf16(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
     const bool pv = A.L.keep_v < kHeadDim;                  // value rows are pruned: expand them per page
     switch (G) {
-        case 1: return pv ? launch_bf16<1, true>(A, n_sms, smem_optin, stream) : launch_bf16<1, false>(A, n_sms, smem_optin, stream);
-        case 2: return pv ? launch_bf16<2, true>(A, n_sms, smem_optin, stream) : launch_bf16<2, false>(A, n_sms, smem_optin, stream);
-        case 3: return pv ? launch_bf16<3, true>(A, n_sms, smem_optin, stream) : launch_bf16<3, false>(A, n_sms, smem_optin, stream);
-        case 4: return pv ? launch_bf16<4, true>(A, n_sms, smem_optin, stream) : launch_bf16<4, false>(A, n_sms, smem_optin, stream);
-        case 5: return pv ? launch_bf16<5, true>(A, n_sms, smem_optin, stream) : launch_bf16<5, false>(A, n_sms, smem_optin, stream);
-        case 6: return pv ? launch_bf16<6, true>(A, n_sms, smem_optin, stream) : launch_bf16<6, false>(A, n_sms, smem_optin, stream);
-        case 7: return pv ? launch_bf16<7, true>(A, n_sms, smem_optin, stream) : launch_bf16<7, false>(A, n_sms, smem_optin, stream);
-        case 8: return pv ? launch_bf16<8, true>(A, n_sms, smem_optin, stream) : launch_bf16<8, false>(A, n_sms, smem_optin, stream);
+        case 1: return pv ? launch_bf16<1, true>(A, dev, info, stream) : launch_bf16<1, false>(A, dev, info, stream);
+        case 2: return pv ? launch_bf16<2, true>(A, dev, info, stream) : launch_bf16<2, false>(A, dev, info, stream);
+        case 3: return pv ? launch_bf16<3, true>(A, dev, info, stream) : launch_bf16<3, false>(A, dev, info, stream);
+        case 4: return pv ? launch_bf16<4, true>(A, dev, info, stream) : launch_bf16<4, false>(A, dev, info, stream);
+        case 5: return pv ? launch_bf16<5, true>(A, dev, info, stream) : launch_bf16<5, false>(A, dev, info, stream);
+        case 6: return pv ? launch_bf16<6, true>(A, dev, info, stream) : launch_bf16<6, false>(A, dev, info, stream);
+        case 7: return pv ? launch_bf16<7, true>(A, dev, info, stream) : launch_bf16<7, false>(A, dev, info, stream);
+        case 8: return pv ? launch_bf16<8, true>(A, dev, info, stream) : launch_bf16<8, false>(A, dev, info, stream);
         default: return SPARK_ERR_UNSUPPORTED;
     }
 }

@@ -53,11 +53,13 @@ extern "C" spark_status spark_decode_attn_noalloc(const spark_params* p, const v
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!q || !pages || !block_table || !packed_lens || !qnorm || !out) return SPARK_ERR_NULL;
+    if (!q || !pages || !packed_lens || !qnorm || !out) return SPARK_ERR_NULL;
     if (max_blocks < 0 || max_blocks > INT32_MAX / kPageTokens) return SPARK_ERR_BAD_SHAPE;
     if ((reinterpret_cast<uintptr_t>(pages) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
         (reinterpret_cast<uintptr_t>(qnorm) & 15) || (reinterpret_cast<uintptr_t>(out) & 15) ||
         (reinterpret_cast<uintptr_t>(lse) & 3))
+        return SPARK_ERR_BAD_SHAPE;
+    if (!block_table && static_cast<int64_t>(p->batch) * p->n_kv_heads * max_blocks > p->n_pool_pages)
         return SPARK_ERR_BAD_SHAPE;
     // the built-in scratch has a fixed size: refuse anything it cannot hold
     if (static_cast<int64_t>(p->batch) * p->n_kv_heads > kNoAllocMaxUnits ||

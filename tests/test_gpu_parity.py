@@ -203,7 +203,8 @@ def test_config2_llama_32k_full():
 
 def test_bad_page_id_is_recorded_not_dereferenced():
     wl = make("bf16", 1, 4, 1, [64], 4, 64, seed=110, gap=False)
-    cache = SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype="bf16", max_tokens=64)
+    cache = SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=4, keep=64, dtype="bf16", max_tokens=64,
+                       block_table=B.identity_block_table(1, 1, 4, "cuda"))
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     assert cache.status() == 0
     cache.block_table[0, 0, 1] = 1 << 20                       # outside the pool

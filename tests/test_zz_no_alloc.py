@@ -37,8 +37,10 @@ def built():
 def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, keep, keep_v):
     wl = inputs.make_workload(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=lens, window=16, dtype=dtype,
                               sigma_s=1.0 if dtype == "bf16" else 0.5, seed=321, device="cuda")
+    # one case with an explicit block table, the others contiguous (no table)
+    table = B.identity_block_table(Bn, Hkv, (max(lens) + 15) // 16, "cuda") if keep == 38 else None
     cache = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=16, keep=keep, dtype=dtype,
-                       max_tokens=max(lens), keep_v=keep_v)
+                       max_tokens=max(lens), keep_v=keep_v, block_table=table)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     lse_ref = torch.empty(Bn, Hq, dtype=torch.float32, device="cuda")
     ref = cache.decode(wl.q, lse=lse_ref)
@@ -53,7 +55,7 @@ def test_noalloc_matches_regular_entry_point_twice(dtype, Bn, Hq, Hkv, lens, kee
         out = torch.full((Bn, Hq, 128), float("nan"), dtype=torch.float32, device="cuda")
         lse = torch.full((Bn, Hq), float("nan"), dtype=torch.float32, device="cuda")
         B.spark_decode_attn_noalloc(cache.params, wl.q, cache.pages, cache.block_table, cache.packed_lens,
-                                    cache.qnorm, out, lse)
+                                    cache.qnorm, out, lse, max_blocks=cache.table_blocks)
         torch.cuda.synchronize()
         d = float((out - ref).abs().max())
         assert d <= TOL[dtype], f"call {call}: max|delta| {d:.3e}"

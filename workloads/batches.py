@@ -42,6 +42,8 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
     batch = SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
                        max_tokens=min(S, budget), device=device, flags=flags, keep_v=keep_v, guard=guard)
     blocks = batch.max_blocks
+    from paper_2508_15212_b200 import binding as B
+    rows = B.identity_block_table(Bn, Hkv, blocks, device)     # where each prompt's pages sit in the batch pool
     qs, kept, dense = [], [], {}
     batch.prep_us = []                     # evict + prune time of each prompt (CUDA events)
     for b in range(Bn):
@@ -50,7 +52,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
                                   seed=int(config["seed"]) + 7 * b + 1000003 * seed_offset, device=device)
         one = SparkCache(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=config["dtype"],
                          max_tokens=S, device=device, token_budget=budget, pool_kernel=pool,
-                         block_table=batch.block_table[b:b + 1].contiguous(),
+                         block_table=rows[b:b + 1].contiguous(),
                          n_pool_pages=batch.params.n_pool_pages, pages=batch.pages, keep_v=keep_v)
         assert one.block_table.shape[-1] == blocks
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
