@@ -21,11 +21,11 @@ constexpr int kStepTokens = 2 * kPageTokens;              // a lane per token: t
 template <int G> struct SmemF32 {
     static constexpr int GP = ((G + 1 + 3) / 4) * 4;     // floats per table entry: G scaled queries + 1/a
     static constexpr int GPP = ((G + 3) / 4) * 4;        // floats per probability entry
-    static constexpr int kQtab = kCtrlBytes + kPrefixBytes;
+    static constexpr int kQtab = kCtrlBytes;
     static constexpr int kQsum = kQtab + kHeadDim * GP * 4;
     static constexpr int kPscr = kQsum + 32;
     static constexpr int kMerge = kPscr + kConsumerWarps * 32 * GPP * 4;
-    static constexpr int kRing = (kMerge + merge_bytes(kConsumerWarps, G) + 127) / 128 * 128;
+    static constexpr int kFixed = (kMerge + merge_bytes(kConsumerWarps, G) + 127) / 128 * 128;   // prefix and ring start here
 };
 
 template <int G>
@@ -34,12 +34,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
     using S = SmemF32<G>;
     constexpr int GP = S::GP, GPP = S::GPP;
     extern __shared__ __align__(128) unsigned char smem[];
-    const Ctrl C = make_ctrl(smem);
+    const Ctrl C = make_ctrl(smem, A.prefix_off);
     float* qtab = reinterpret_cast<float*>(smem + S::kQtab);
     float* qsum = reinterpret_cast<float*>(smem + S::kQsum);
     float* pscr_all = reinterpret_cast<float*>(smem + S::kPscr);
     float* merge = reinterpret_cast<float*>(smem + S::kMerge);
-    unsigned char* ring = smem + S::kRing;
+    unsigned char* ring = smem + A.ring_off;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const PageLayout L = A.L;
@@ -266,11 +266,13 @@ static spark_status launch_f32(const DecodeArgs& A0, int dev, const DeviceInfo& 
     using S = SmemF32<G>;
     A.pps = 2;
     A.slot_stride = static_cast<int>(align_up(2 * static_cast<size_t>(A.L.page_bytes), 128));
-    int ns = (smem_optin - S::kRing) / A.slot_stride;
+    A.prefix_off = S::kFixed;
+    A.ring_off = S::kFixed + prefix_bytes(A.B);
+    int ns = (smem_optin - A.ring_off) / A.slot_stride;
     if (ns > kMaxSlots) ns = kMaxSlots;
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
-    const size_t smem = S::kRing + static_cast<size_t>(ns) * A.slot_stride;
+    const size_t smem = A.ring_off + static_cast<size_t>(ns) * A.slot_stride;
     if (!allow_max_smem(decode_f32_kernel<G>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
     return launch_decode_kernel(decode_f32_kernel<G>, grid, kDecodeThreads, smem, stream, A) == cudaSuccess
@@ -314,7 +316,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.status = reinterpret_cast<int*>(ws);
     A.tickets = reinterpret_cast<int*>(ws + kWorkspaceHeader);
     A.partials = reinterpret_cast<float*>(ws + kWorkspaceHeader + align_up(units * sizeof(int), 256));
-    A.nslots = 0; A.slot_stride = 0; A.pps = 1;
+    A.nslots = 0; A.slot_stride = 0; A.pps = 1; A.prefix_off = 0; A.ring_off = 0;
     A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
     const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, dev, info, stream)
                                                     : launch_decode_f32(G, A, dev, info, stream);

@@ -40,24 +40,26 @@ struct DecodeArgs {
     int nslots;
     int slot_stride;
     int pps;                                 // pages per step (= per ring slot): 1 or 2
+    int prefix_off;                          // shared-memory offset of the steps-per-sequence prefix ((B + 1) ints)
+    int ring_off;                            // shared-memory offset of the ring (behind the prefix)
     int overlap;                             // launched as a programmatic dependent of the preceding kernel
 };
 
 // control block at the start of dynamic shared memory
 constexpr int kCtrlBytes = 1024;                                 // full[32], empty[32], flags, plan
-constexpr int kPrefixBytes = ((kMaxBatch + 1) * 4 + 15) / 16 * 16;
+// the steps-per-sequence prefix sits between a kernel's fixed shared-memory areas and the ring and is as
+// large as the batch needs, so small batches leave its room to the ring
+inline int prefix_bytes(int batch) { return ((batch + 1) * 4 + 127) / 128 * 128; }
 
-// Shared merge area for `nw` consumer warps and `g` heads: the warps' states ([warp][head][kRec] floats),
-// reused by the final combine for the weights of up to kMaxCtas parts, the heads' (M, L) and one float4
-// per consumer thread; behind it the weights of the warps ([head][32]) and the heads' (M, L).
+// Shared merge area for `nw` consumer warps and `g` heads: the warps' states ([warp][head][kRec] floats:
+// 128 outputs, m, l and two spare words that the CTA-wide merge uses for the warp's weight and the head's
+// (M, L)), reused by the final combine for the weights of up to kMaxCtas parts, the heads' (M, L) and one
+// float4 per consumer thread.
 __host__ __device__ constexpr int merge_state_floats(int nw, int g)
 {
     return nw * g * kRec > kMaxCtas * g * 2 + nw * 32 * 4 ? nw * g * kRec : kMaxCtas * g * 2 + nw * 32 * 4;
 }
-__host__ __device__ constexpr int merge_bytes(int nw, int g)
-{
-    return (merge_state_floats(nw, g) + g * 32 + g * 2 + 2) * 4;
-}
+__host__ __device__ constexpr int merge_bytes(int nw, int g) { return merge_state_floats(nw, g) * 4; }
 
 // ---- PTX helpers ----------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void* p)
@@ -245,7 +247,7 @@ struct Ctrl {
     int* prefix;
 };
 
-__device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
+__device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem, int prefix_off)
 {
     Ctrl c;
     c.full = reinterpret_cast<uint64_t*>(smem);
@@ -254,7 +256,7 @@ __device__ __forceinline__ Ctrl make_ctrl(unsigned char* smem)
     c.last_flag = reinterpret_cast<volatile int*>(smem + 516);
     c.plan = reinterpret_cast<Plan*>(smem + 528);
     c.seq = reinterpret_cast<volatile int*>(smem + 640);
-    c.prefix = reinterpret_cast<int*>(smem + kCtrlBytes);
+    c.prefix = reinterpret_cast<int*>(smem + prefix_off);
     return c;
 }
 
@@ -501,8 +503,8 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
     int first_cta, n_parts;
     unit_parts(*C.plan, sg.unit_start, sg.steps_b, first_cta, n_parts);
     const int unit = b * A.Hkv + h;
-    float* wts = merge + merge_state_floats(NW, G);           // [G][32] weights of the warps, then [G][2] (M, L)
-    float* ML = wts + G * 32;
+    static_assert(NW >= 2, "the heads' (M, L) live in the spare words of the first two warps' records");
+    constexpr int kWt = kHeadDim + 2, kMl = kHeadDim + 3;     // spare words of a record
     // ---- weights of the warps: warp g serves head g, lane w holds warp w's (m, l) ----
     if (warp < G) {
         const float m = lane < NW ? merge[(lane * G + warp) * kRec + kHeadDim] : -INFINITY;
@@ -514,8 +516,8 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
         float Ls = l * wt;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(kFull, Ls, o);
-        wts[warp * 32 + lane] = wt;
-        if (lane == 0) { ML[2 * warp] = M; ML[2 * warp + 1] = Ls; }
+        if (lane < NW) merge[(lane * G + warp) * kRec + kWt] = wt;
+        if (lane == 0) { merge[warp * kRec + kMl] = M; merge[(G + warp) * kRec + kMl] = Ls; }
     }
     consumer_sync<NT>();
     // ---- weighted sums: a thread owns two channels of one head ----
@@ -528,11 +530,11 @@ __device__ __forceinline__ void merge_and_publish(const DecodeArgs& A, const Ctr
         float2 O = make_float2(0.f, 0.f);
 #pragma unroll
         for (int w = 0; w < NW; ++w) {
-            const float f = wts[gg * 32 + w];
+            const float f = merge[(w * G + gg) * kRec + kWt];
             O.x = fmaf(v[w].x, f, O.x);
             O.y = fmaf(v[w].y, f, O.y);
         }
-        const float M = ML[2 * gg], Ls = ML[2 * gg + 1];
+        const float M = merge[gg * kRec + kMl], Ls = merge[(G + gg) * kRec + kMl];
         if (n_parts == 1) {
             const float inv = 1.0f / Ls;
             *reinterpret_cast<float2*>(A.out + (static_cast<int64_t>(b) * A.Hq + h * G + gg) * kHeadDim + 2 * c2) =

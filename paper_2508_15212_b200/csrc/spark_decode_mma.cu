@@ -35,12 +35,13 @@ constexpr float kSlack = 8.f;                 // log2 units a score may exceed t
 
 constexpr int kVTileBytes = kPageTokens * kHeadDim * 2;                          // dense value rows of one page
 
+// Shared-memory map (fixed part; the steps prefix and the ring follow at offsets chosen by the launcher).
 template <int G, bool kPV> struct SmemBf16 {
-    static constexpr int kTab = kCtrlBytes + kPrefixBytes;                       // q, q' high, q' low: 3 x [G][128] bf16
+    static constexpr int kTab = kCtrlBytes;                                      // q, q' high, q' low: 3 x [G][128] bf16
     static constexpr int kQsum = kTab + 3 * G * kHeadDim * 2;                    // [8] float
     static constexpr int kMerge = kQsum + 32;
     static constexpr int kVTile = (kMerge + merge_bytes(kNW, G) + 127) / 128 * 128;   // per-warp tiles (pruned values)
-    static constexpr int kRing = kVTile + (kPV ? kNW * kVTileBytes : 0);
+    static constexpr int kFixed = kVTile + (kPV ? kNW * kVTileBytes : 0);        // prefix and ring start here
 };
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -184,6 +185,33 @@ __device__ __forceinline__ void expand_nibble_v(unsigned w, unsigned b0m, unsign
         : "r"(w), "r"(b0m), "r"(b1m), "r"(b2m), "r"(b3m));
 }
 
+// Tables of one query head of a unit (one warp; lane l owns channels 4l .. 4l+3):
+//   tab[0][hd][j] = q[j] (bf16 as stored), tab[1] / tab[2] = bf16 high / low part of q[j] / a[j],
+//   qsum[hd]      = sum over all 128 channels of the 16-bit q' (so kept terms cancel exactly).
+template <int G>
+__device__ __forceinline__ void write_head_tables(unsigned char* tab, float* qsum, int hd, int lane, uint2 qr, float4 a4)
+{
+    const float qf[4] = {__uint_as_float(qr.x << 16), __uint_as_float(qr.x & 0xffff0000u),
+                         __uint_as_float(qr.y << 16), __uint_as_float(qr.y & 0xffff0000u)};
+    const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+    float hi[4], lo[4];
+    double part = 0.0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float qp = qf[e] / av[e];
+        hi[e] = bf16_round(qp);
+        lo[e] = bf16_round(qp - hi[e]);
+        part += static_cast<double>(hi[e]) + static_cast<double>(lo[e]);
+    }
+    unsigned char* row = tab + hd * (kHeadDim * 2) + lane * 8;
+    *reinterpret_cast<uint2*>(row) = qr;
+    *reinterpret_cast<uint2*>(row + G * kHeadDim * 2) = make_uint2(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]));
+    *reinterpret_cast<uint2*>(row + 2 * G * kHeadDim * 2) = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFull, part, o);
+    if (lane == 0) qsum[hd] = static_cast<float>(part);
+}
+
 __device__ __forceinline__ void sts_u32x4(unsigned addr, unsigned a, unsigned b, unsigned c, unsigned d)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -195,11 +223,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
     using S = SmemBf16<G, kPV>;
     constexpr bool kShared8 = (G <= 4);        // q' high and low parts share one 8-column operand
     extern __shared__ __align__(128) unsigned char smem[];
-    const Ctrl C = make_ctrl(smem);
+    const Ctrl C = make_ctrl(smem, A.prefix_off);
     unsigned char* tab = smem + S::kTab;
     float* qsum_s = reinterpret_cast<float*>(smem + S::kQsum);
     float* merge = reinterpret_cast<float*>(smem + S::kMerge);
-    unsigned char* ring = smem + S::kRing;
+    unsigned char* ring = smem + A.ring_off;
     const unsigned ring_u = smem_u32(ring);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -231,33 +259,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
         const int len = clamp_len(A.lens[b], max_tokens);
 
         // ---- per-unit tables, built once per CTA: warp `hd` prepares query head hd ----
-        //   tab[0][hd][j] = q[j] (bf16 as stored), tab[1] / tab[2] = bf16 high / low part of q[j] / a[j],
-        //   qsum_s[hd]    = sum over all 128 channels of the 16-bit q' (so kept terms cancel exactly).
         if (warp < G) {
             const uint2 qr = *reinterpret_cast<const uint2*>(
                 static_cast<const unsigned short*>(A.q) +
                 (static_cast<int64_t>(b) * A.Hq + h * G + warp) * kHeadDim + 4 * lane);
             const float4 a4 = *reinterpret_cast<const float4*>(
                 A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + 4 * lane);
-            const float qf[4] = {__uint_as_float(qr.x << 16), __uint_as_float(qr.x & 0xffff0000u),
-                                 __uint_as_float(qr.y << 16), __uint_as_float(qr.y & 0xffff0000u)};
-            const float av[4] = {a4.x, a4.y, a4.z, a4.w};
-            float hi[4], lo[4];
-            double part = 0.0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float qp = qf[e] / av[e];
-                hi[e] = bf16_round(qp);
-                lo[e] = bf16_round(qp - hi[e]);
-                part += static_cast<double>(hi[e]) + static_cast<double>(lo[e]);
-            }
-            unsigned char* row = tab + warp * (kHeadDim * 2) + lane * 8;
-            *reinterpret_cast<uint2*>(row) = qr;
-            *reinterpret_cast<uint2*>(row + G * kHeadDim * 2) = make_uint2(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]));
-            *reinterpret_cast<uint2*>(row + 2 * G * kHeadDim * 2) = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFull, part, o);
-            if (lane == 0) qsum_s[warp] = static_cast<float>(part);
+            write_head_tables<G>(tab, qsum_s, warp, lane, qr, a4);
         }
         consumer_sync<kNT>();
         // second-operand fragments (column r of each operand, channels 32c .. 32c+31):
@@ -485,11 +493,13 @@ static spark_status launch_bf16(const DecodeArgs& A0, int dev, const DeviceInfo&
     using S = SmemBf16<G, kPV>;
     A.pps = 1;
     A.slot_stride = static_cast<int>(align_up(static_cast<size_t>(A.L.page_bytes), 128));
-    int ns = (smem_optin - S::kRing) / A.slot_stride;
+    A.prefix_off = S::kFixed;
+    A.ring_off = S::kFixed + prefix_bytes(A.B);
+    int ns = (smem_optin - A.ring_off) / A.slot_stride;
     if (ns > kMaxSlots) ns = kMaxSlots;
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
-    const size_t smem = S::kRing + static_cast<size_t>(ns) * A.slot_stride;
+    const size_t smem = A.ring_off + static_cast<size_t>(ns) * A.slot_stride;
     if (!allow_max_smem(decode_bf16_kernel<G, kPV>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
     return launch_decode_kernel(decode_bf16_kernel<G, kPV>, grid, kThreads, smem, stream, A) == cudaSuccess
