@@ -18,6 +18,9 @@
  *     status word at the start of the workspace and the kernel returns without
  *     touching the bad address; read them with spark_read_status.
  *   - head_dim must be 128, page_tokens 16, 1 <= n_q_heads / n_kv_heads <= 8.
+ *   - Alignment: q, k_new, v_new, qnorm, out and the page pool must be 16-byte aligned (the kernels use
+ *     16-byte vector accesses), workspaces 256-byte aligned; a misaligned pointer is refused with
+ *     SPARK_ERR_BAD_SHAPE.  max_blocks must not exceed INT32_MAX / 16.
  *
  * Packed cache.  The cache is a pool of fixed-size pages.  One page holds
  * `page_tokens` consecutive tokens of ONE KV head of one sequence:
@@ -26,7 +29,10 @@
  * or, with value-channel pruning (keep_v < head_dim), kept value entries and a second
  * 128-bit mask per token in place of the dense value rows.
  * `block_table[b][h][i]` is the pool index of the page with tokens
- * [16 i, 16 i + 16) of sequence b, KV head h.  The byte layout inside a page is
+ * [16 i, 16 i + 16) of sequence b, KV head h.  Every call that takes a block table also accepts NULL for a
+ * CONTIGUOUS cache: unit (b, h) then owns the max_blocks consecutive pages starting at
+ * (b * n_kv_heads + h) * max_blocks, n_pool_pages must cover them all, and the decode step saves the table
+ * lookups.  The byte layout inside a page is
  * private to the library (spark_page_bytes gives its size; spark_unpack_pages
  * turns pages back into logical arrays).  Slots of a page past the end of the
  * sequence are zero.
@@ -195,6 +201,26 @@ spark_status spark_decode_attn(const spark_params *p, const void *q,
                                const int32_t *packed_lens, const float *qnorm,
                                float *out, float *lse,
                                void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
+ * spark_decode_attn_host -- the same decode step for a caller whose query and result live in HOST memory
+ * (Sec. "Channel Recovery" / "Preliminaries" as above; only the transport differs).  Enqueues, in this order
+ * on `stream`: the copy of q_host to q_dev, spark_decode_attn on q_dev, the copy of out_dev to out_host (and
+ * of lse_dev to lse_host when both are given).  Nothing is synchronised: the results are in out_host once
+ * the stream has reached this point.
+ *
+ *   q_host             HOST [B][Hq][D], dtype as the cache; page-locked memory lets the copy run asynchronously
+ *   q_dev              DEVICE staging for the query, same size, 16-byte aligned
+ *   out_dev            DEVICE [B][Hq][D] fp32, 16-byte aligned;  out_host  HOST, same size
+ *   lse_dev, lse_host  optional, both NULL or both given, [B][Hq] fp32
+ *   every other argument as for spark_decode_attn; errors are returned before anything is enqueued
+ *   except a failing copy (SPARK_ERR_CUDA).
+ */
+spark_status spark_decode_attn_host(const spark_params *p, const void *q_host, void *q_dev,
+                                    const void *pages, const int32_t *block_table, int32_t max_blocks,
+                                    const int32_t *packed_lens, const float *qnorm,
+                                    float *out_dev, float *out_host, float *lse_dev, float *lse_host,
+                                    void *workspace, size_t workspace_bytes, spark_stream_t stream);
 
 /*
  * spark_decode_attn_noalloc -- spark_decode_attn for callers that cannot allocate device memory.

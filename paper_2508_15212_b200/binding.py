@@ -22,7 +22,7 @@ SPARK_F32, SPARK_BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
-           "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_noalloc", "spark_unpack_pages",
+           "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_host", "spark_decode_attn_noalloc", "spark_unpack_pages",
            "spark_unpack_value_masks", "spark_read_status"]
 
 
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.spark_append.argtypes = [P, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.spark_decode_attn.restype = i32
         L.spark_decode_attn.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spark_decode_attn_host.restype = i32
+        L.spark_decode_attn_host.argtypes = [P, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.spark_decode_attn_noalloc.restype = i32
         L.spark_decode_attn_noalloc.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.spark_unpack_pages.restype = i32
@@ -175,6 +177,52 @@ def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm
                                    _blocks(block_table, max_blocks), _ptr(packed_lens), _ptr(qnorm), _ptr(out), _ptr(lse),
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
            "spark_decode_attn")
+
+
+class BoundDecodeHost:
+    """spark_decode_attn_host with every argument marshalled once: query and result in page-locked host
+    tensors, device staging owned by this object's caller.  Calling it enqueues copy-in, the step and
+    copy-out on the stream; it does not synchronise."""
+
+    def __init__(self, p: spark_params, q_host, q_dev, pages, block_table, packed_lens, qnorm, out_dev, out_host,
+                 workspace, max_blocks=None, stream: Optional[int] = None):
+        assert q_host.is_pinned() and out_host.is_pinned() and q_host.is_contiguous() and out_host.is_contiguous()
+        self._alive = (p, q_host, q_dev, pages, block_table, packed_lens, qnorm, out_dev, out_host, workspace)
+        self._fn = lib().spark_decode_attn_host
+        self._args = (ctypes.byref(p), _ptr(q_host), _ptr(q_dev), _ptr(pages), _ptr(block_table),
+                      _blocks(block_table, max_blocks), _ptr(packed_lens), _ptr(qnorm), _ptr(out_dev), _ptr(out_host),
+                      None, None, _ptr(workspace), workspace.numel() * workspace.element_size())
+        self._stream = None if stream is None else ctypes.c_void_p(stream)
+        self.out_host = out_host
+
+    def __call__(self) -> None:
+        code = self._fn(*self._args, self._stream if self._stream is not None else _stream())
+        if code != SPARK_OK:
+            raise SparkError(code, "spark_decode_attn_host")
+
+
+class BoundDecode:
+    """spark_decode_attn with every argument marshalled once.
+
+    A decode loop calls the same entry point with the same buffers step after step; this object converts
+    the pointers and sizes to C values a single time, so a call costs one foreign-function call (the
+    stream is the only thing looked up per call, unless a fixed stream handle is given).
+    """
+
+    def __init__(self, p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse, workspace,
+                 max_blocks=None, stream: Optional[int] = None):
+        self._alive = (p, q, pages, block_table, packed_lens, qnorm, out, lse, workspace)     # keep the buffers
+        self._fn = lib().spark_decode_attn
+        self._args = (ctypes.byref(p), _ptr(q), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
+                      _ptr(packed_lens), _ptr(qnorm), _ptr(out), _ptr(lse), _ptr(workspace),
+                      workspace.numel() * workspace.element_size())
+        self._stream = None if stream is None else ctypes.c_void_p(stream)
+        self.out = out
+
+    def __call__(self) -> None:
+        code = self._fn(*self._args, self._stream if self._stream is not None else _stream())
+        if code != SPARK_OK:
+            raise SparkError(code, "spark_decode_attn")
 
 
 def spark_decode_attn_noalloc(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse,

@@ -107,6 +107,22 @@ class SparkCache:
                             self.ws_decode, max_blocks=self.table_blocks)
         return out
 
+    def bind_decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                    stream: Optional[int] = None) -> "B.BoundDecode":
+        """The decode step on fixed buffers, marshalled once (for decode loops); call the result to enqueue it."""
+        if out is None:
+            out = self.alloc_out()
+        return B.BoundDecode(self.params, q, self.pages, self.block_table, self.packed_lens, self.qnorm, out, lse,
+                             self.ws_decode, max_blocks=self.table_blocks, stream=stream)
+
+    def bind_decode_host(self, q_host, out_host, stream: Optional[int] = None) -> "B.BoundDecodeHost":
+        """The decode step for a query and a result in page-locked host tensors (copy-in, step, copy-out in one
+        call, nothing synchronised); the device staging buffers are allocated here, once."""
+        q_dev = torch.empty(q_host.shape, dtype=q_host.dtype, device=self.device)
+        return B.BoundDecodeHost(self.params, q_host, q_dev, self.pages, self.block_table, self.packed_lens,
+                                 self.qnorm, self.alloc_out(), out_host, self.ws_decode,
+                                 max_blocks=self.table_blocks, stream=stream)
+
     # -- inspection ------------------------------------------------------------------------------
     def unpack(self, want_vals=True, want_v=True, want_vmask=False) -> Dict[str, torch.Tensor]:
         p, n = self.params, self.max_tokens

@@ -167,6 +167,31 @@ spark_status spark_decode_attn(const spark_params* p, const void* q, const void*
     return st;
 }
 
+spark_status spark_decode_attn_host(const spark_params* p, const void* q_host, void* q_dev, const void* pages,
+                                    const int32_t* block_table, int32_t max_blocks,
+                                    const int32_t* packed_lens, const float* qnorm, float* out_dev,
+                                    float* out_host, float* lse_dev, float* lse_host, void* workspace,
+                                    size_t workspace_bytes, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!q_host || !q_dev || !out_dev || !out_host) return SPARK_ERR_NULL;
+    if ((lse_dev == nullptr) != (lse_host == nullptr)) return SPARK_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t e = (p->dtype == SPARK_BF16) ? 2 : 4;
+    const size_t nq = static_cast<size_t>(p->batch) * p->n_q_heads * p->head_dim;
+    if (cudaMemcpyAsync(q_dev, q_host, nq * e, cudaMemcpyHostToDevice, s) != cudaSuccess) return SPARK_ERR_CUDA;
+    st = spark_decode_attn(p, q_dev, pages, block_table, max_blocks, packed_lens, qnorm, out_dev, lse_dev,
+                           workspace, workspace_bytes, stream);
+    if (st != SPARK_OK) return st;
+    if (cudaMemcpyAsync(out_host, out_dev, nq * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    if (lse_dev && cudaMemcpyAsync(lse_host, lse_dev, static_cast<size_t>(p->batch) * p->n_q_heads * sizeof(float),
+                                   cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    return SPARK_OK;
+}
+
 spark_status spark_unpack_pages(const spark_params* p, const void* pages, const int32_t* block_table,
                                 int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
                                 uint32_t* mask, float* mu, void* vals, void* v, spark_stream_t stream)

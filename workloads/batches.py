@@ -31,11 +31,13 @@ def permuted_block_table(batch: int, n_kv_heads: int, lens, device, seed: int, s
 
 def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int = None, seed_offset: int = 0,
                         keep_prompts=(), flags: int = 0, keep_v: int = 0,
-                        guard: bool = False):
+                        guard: bool = False, keep_gathered: bool = False):
     """Configuration 4: prompts are generated, evicted to the token budget and pruned ONE AT A TIME (each
     prompt's dense K/V is freed before the next), into one shared page pool; the result is a batch cache
     whose decode step serves all prompts.  Returns (cache, q [B,Hq,D], kept_tokens [B,Hkv,budget], dense)
-    where `dense` maps each prompt index listed in `keep_prompts` to its dense workload, for checks."""
+    where `dense` maps each prompt index listed in `keep_prompts` to its dense workload, for checks.  With
+    `keep_gathered` the cache also carries `gathered = (q_win, k, v)`: every prompt's window queries and the keys
+    and values of its kept tokens ([B,Hkv,budget,D]), the input an oracle needs to redo pruning and decode."""
     Bn = int(n_prompts or config["batch"])
     Hq, Hkv, W, S = config["n_q_heads"], config["n_kv_heads"], config["window"], int(config["seq_lens"])
     budget, pool = int(config["token_budget"]), int(config["pool_kernel"])
@@ -45,6 +47,7 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
     from paper_2508_15212_b200 import binding as B
     rows = B.identity_block_table(Bn, Hkv, blocks, device)     # where each prompt's pages sit in the batch pool
     qs, kept, dense = [], [], {}
+    gath = ([], [], []) if keep_gathered else None
     batch.prep_us = []                     # evict + prune time of each prompt (CUDA events)
     for b in range(Bn):
         wl = inputs.make_workload(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, seq_lens=S, window=W,
@@ -68,5 +71,11 @@ def build_evicted_batch(config: dict, keep: int, device="cuda", n_prompts: int =
         assert one.status() == 0
         if b in keep_prompts:
             dense[b] = wl
+        if keep_gathered:
+            idx = one.kept_tokens[0].long().unsqueeze(-1).expand(Hkv, budget, 128)
+            gath[0].append(wl.q_win[0])
+            gath[1].append(wl.k[0].gather(1, idx))
+            gath[2].append(wl.v[0].gather(1, idx))
         del wl, one
+    batch.gathered = tuple(torch.stack(x) for x in gath) if keep_gathered else None
     return batch, torch.stack(qs), torch.stack(kept), dense
