@@ -194,3 +194,75 @@ def evict(q_win, k, seq_lens, budget: int, pool: int = 7, *, want_votes: bool = 
                             int(pool), _ptr(kept), _ptr(out_len), _ptr(vote), _ptr(pooled))
     assert rc == 0, rc
     return (kept, out_len, vote, pooled) if want_votes else (kept, out_len)
+
+
+def select_variant(k, seq_lens, a, *, top_p: float = None, cap: int = None, group_prune=None, want_stats=False):
+    """Adaptive selection (Sec. "Ablation Studies"): SparK-p when `top_p` is given (at most `cap` channels),
+    SparK-g when `group_prune` (ratios from the most salient rank group to the least) is given.
+    -> dict(mask, mu, count[, mu_all, sigma_all])"""
+    kk, dt = _as_np(k)
+    B, Hkv, S, D = kk.shape
+    sb, sh, st = _kv_strides(kk)
+    lens = _i32(seq_lens)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    MW = (D + 31) // 32
+    mask = np.empty((B, Hkv, S, MW), np.uint32)
+    mu = np.empty((B, Hkv, S), np.float32)
+    count = np.empty((B, Hkv, S), np.int32)
+    mu_all = np.empty((B, Hkv, S), np.float32) if want_stats else None
+    sg_all = np.empty((B, Hkv, S), np.float32) if want_stats else None
+    assert (top_p is None) != (group_prune is None)
+    if top_p is not None:
+        variant, n_groups, prune = 1, 0, None
+        cap = D if cap is None else int(cap)
+    else:
+        variant, top_p, cap = 2, 0.0, D
+        prune = np.ascontiguousarray(group_prune, dtype=np.float32)
+        n_groups = int(prune.size)
+    rc = lib().oracle_select_variant(_ptr(kk), dt, B, Hkv, D, ctypes.c_int64(sb), ctypes.c_int64(sh),
+                                     ctypes.c_int64(st), _ptr(lens), S, _ptr(a), variant,
+                                     ctypes.c_float(top_p), int(cap), n_groups, _ptr(prune), _ptr(mask),
+                                     _ptr(mu), _ptr(count), _ptr(mu_all), _ptr(sg_all))
+    assert rc == 0, rc
+    out = dict(mask=mask, mu=mu, count=count)
+    if want_stats:
+        out["mu_all"], out["sigma_all"] = mu_all, sg_all
+    return out
+
+
+def draw_uniforms(seed: int, unit: int, t: int, j: int):
+    """The two 24-bit uniforms of the sampled-recovery draw of entry (unit, t, j)."""
+    u1, u2 = ctypes.c_double(0), ctypes.c_double(0)
+    lib().oracle_draw_uniforms(ctypes.c_uint32(seed), ctypes.c_int64(unit), ctypes.c_int64(t), int(j),
+                               ctypes.byref(u1), ctypes.byref(u2))
+    return u1.value, u2.value
+
+
+def decode_attn_sampled(q, k, v, lens, mask, mu_all, sigma_all, a, *, mode: int, seed: int, scale: float = 0.0,
+                        want_recovered: bool = False):
+    """Sec. "Channel Recovery" with a Gaussian (mode 1) or Exponential (mode 2) recovery distribution.
+    -> (out, lse[, recovered saliencies [B,Hkv,S,D] float64])"""
+    qq, dtq = _as_np(q)
+    kk, dt = _as_np(k)
+    vv, dtv = _as_np(v)
+    assert dtq == dt == dtv
+    qq = np.ascontiguousarray(qq)
+    B, Hkv, S, D = kk.shape
+    Hq = qq.shape[1]
+    sb, sh, st = _kv_strides(kk)
+    assert _kv_strides(vv) == (sb, sh, st)
+    lens = _i32(lens)
+    mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    mu_all = np.ascontiguousarray(mu_all, dtype=np.float32)
+    sigma_all = None if sigma_all is None else np.ascontiguousarray(sigma_all, dtype=np.float32)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    out = np.empty((B, Hq, D), np.float32)
+    lse = np.empty((B, Hq), np.float32)
+    rec = np.zeros((B, Hkv, S, D), np.float64) if want_recovered else None
+    rc = lib().oracle_decode_attn_sampled(_ptr(qq), _ptr(kk), _ptr(vv), dt, B, Hq, Hkv, D,
+                                          ctypes.c_int64(sb), ctypes.c_int64(sh), ctypes.c_int64(st),
+                                          _ptr(lens), S, _ptr(mask), _ptr(mu_all), _ptr(sigma_all), _ptr(a),
+                                          ctypes.c_double(scale), int(mode), ctypes.c_uint32(seed),
+                                          _ptr(out), _ptr(lse), _ptr(rec))
+    assert rc == 0, rc
+    return (out, lse, rec) if want_recovered else (out, lse)

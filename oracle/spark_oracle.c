@@ -24,6 +24,13 @@
  *   value-channel pruning ..... App. "Pruning Value Cache Channels": per token, the T_v value
  *                               channels of largest magnitude are kept; the rest are removed
  *
+ *   adaptive variants ......... Sec. "Ablation Studies", "Adaptive Variants": SparK-p keeps, per token, the
+ *                               fewest most salient channels whose saliency adds up to a fraction p of the
+ *                               token's total; SparK-g cuts the channels, ranked by saliency, into g groups
+ *                               and prunes the less salient groups harder
+ *   sampled recovery .......... Sec. "Channel Recovery": w~ ~ N(mu, sigma^2) or w~ ~ Exp(1/mu) with the
+ *                               all-channel statistics of App. "Caching Pruned Channel Statistics"
+ *
  * Readings taken where the paper is silent (each listed in the design notes):
  *   - ||q-bar^j||_2 of a scalar channel is |q-bar^j|; under GQA the G*W window
  *     queries that share a KV head are pooled into one mean;
@@ -35,6 +42,16 @@
  *   - a pruned value entry contributes nothing to the weighted sum (the appendix says value
  *     "recovery requires no additional operations"); the importance of a scalar channel is
  *     its absolute value; ties keep the lower channel.
+ *
+ *   - SparK-p: the running sum and the total are taken in double in rank order (most salient first);
+ *     at least one channel is kept; a page capacity may cap the count;
+ *   - SparK-g: the groups are per-token RANK segments of near-equal size (D / g, the remainder spread over
+ *     the most salient groups); group i keeps its floor((1 - rho_i) n_i) most salient channels, rho listed
+ *     from the most salient group to the least.  (No reading reproduces the overall ratios 0.44 / 0.55 the
+ *     paper's variants table prints beside the listed ratios; this one gives 0.625 / 0.51 at D = 128.)
+ *   - sampled recovery: one draw per pruned entry, a pure function of (seed, sequence, KV head, token,
+ *     channel), so it is fixed for the life of the cache and every decode step sees the same keys;
+ *     Gaussian draws are not clamped (a recovered saliency may be negative).
  *
  * Eviction (observation-window attention-score top-k with max pooling) is not
  * defined by the paper, which only cites the base method and its settings
@@ -379,6 +396,195 @@ int oracle_evict(const void *q_win, const void *k, int dtype, int B, int Hq, int
             int n = 0;
             for (int t = 0; t < S; ++t) if (sel[t]) kt[n++] = t;
             free(vote); free(s); free(cand); free(sel);
+        }
+    return err;
+}
+
+
+/* ---------------------------------------------------------------------------------
+ * Adaptive channel selection (Sec. "Ablation Studies", adaptive variants).
+ *   variant 1 (SparK-p): rank the channels of a token by saliency (descending, lower channel first on
+ *       ties); with c_n = sum of the n largest saliencies (double, in rank order) keep the smallest
+ *       n >= 1 with c_n >= p * c_D, at most `cap` channels.
+ *   variant 2 (SparK-g): cut the ranks into n_groups segments of sizes D / g (+1 for the first D % g
+ *       segments); segment i keeps its floor((1 - prune[i]) * size_i) first ranks.
+ * Outputs as oracle_compress: mask, mu (mean saliency of the pruned channels, 0 when none is pruned),
+ * count (optional, [B][Hkv][S_max] kept channels per token), mu_all / sigma_all (optional).
+ * --------------------------------------------------------------------------------- */
+int oracle_select_variant(const void *k, int dtype, int B, int Hkv, int D,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                          const int32_t *seq_lens, int S_max, const float *a,
+                          int variant, float top_p, int cap, int n_groups, const float *prune,
+                          uint32_t *mask, float *mu, int32_t *count, float *mu_all, float *sigma_all)
+{
+    if (!k || !seq_lens || !a || !mask || !mu) return 1;
+    if (variant == 1 && (!(top_p > 0.f) || !(top_p <= 1.f) || cap < 1 || cap > D)) return 1;
+    if (variant == 2 && (n_groups < 1 || n_groups > D || !prune)) return 1;
+    if (variant != 1 && variant != 2) return 1;
+    const int MW = (D + 31) / 32;
+    int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hkv; ++h) {
+            sal_t *row = (sal_t *)malloc(sizeof(sal_t) * (size_t)D);
+            unsigned char *keep = (unsigned char *)malloc((size_t)D);
+            if (!row || !keep) { err = 2; free(row); free(keep); continue; }
+            const float *au = a + ((int64_t)b * Hkv + h) * D;
+            for (int t = 0; t < S_max; ++t) {
+                int64_t u = ((int64_t)b * Hkv + h) * S_max + t;
+                memset(mask + u * MW, 0, sizeof(uint32_t) * (size_t)MW);
+                mu[u] = 0.f;
+                if (count) count[u] = 0;
+                if (mu_all) mu_all[u] = 0.f;
+                if (sigma_all) sigma_all[u] = 0.f;
+                if (t >= seq_lens[b]) continue;
+                const int64_t kb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                for (int j = 0; j < D; ++j) {
+                    float kf = (float)load_elem(k, kb + j, dtype);
+                    row[j].w = au[j] * fabsf(kf);
+                    row[j].j = j;
+                }
+                if (mu_all || sigma_all) {
+                    double s1 = 0.0;
+                    for (int j = 0; j < D; ++j) s1 += (double)row[j].w;
+                    double m = s1 / (double)D, s2 = 0.0;
+                    for (int j = 0; j < D; ++j) { double d = (double)row[j].w - m; s2 += d * d; }
+                    if (mu_all) mu_all[u] = (float)m;
+                    if (sigma_all) sigma_all[u] = (float)sqrt(s2 / (double)D);
+                }
+                qsort(row, (size_t)D, sizeof(sal_t), sal_cmp);
+                memset(keep, 0, (size_t)D);
+                int n_kept = 0;
+                if (variant == 1) {
+                    double total = 0.0;
+                    for (int r = 0; r < D; ++r) total += (double)row[r].w;
+                    const double need = (double)top_p * total;
+                    double run = 0.0;
+                    int n = D;
+                    for (int r = 0; r < D; ++r) {
+                        run += (double)row[r].w;
+                        if (run >= need) { n = r + 1; break; }
+                    }
+                    if (n > cap) n = cap;
+                    for (int r = 0; r < n; ++r) keep[row[r].j] = 1;
+                    n_kept = n;
+                } else {
+                    int start = 0;
+                    for (int i = 0; i < n_groups; ++i) {
+                        const int size = D / n_groups + (i < D % n_groups ? 1 : 0);
+                        const int kp = (int)floor((1.0 - (double)prune[i]) * (double)size + 1e-9);
+                        for (int r = 0; r < kp && r < size; ++r) keep[row[start + r].j] = 1;
+                        n_kept += kp < size ? (kp > 0 ? kp : 0) : size;
+                        start += size;
+                    }
+                }
+                double pruned_sum = 0.0;
+                for (int r = 0; r < D; ++r) if (!keep[row[r].j]) pruned_sum += (double)row[r].w;
+                mu[u] = (n_kept < D) ? (float)(pruned_sum / (double)(D - n_kept)) : 0.f;
+                if (count) count[u] = n_kept;
+                for (int j = 0; j < D; ++j)
+                    if (keep[j]) mask[u * MW + j / 32] |= (uint32_t)1 << (j % 32);
+            }
+            free(row);
+            free(keep);
+        }
+    return err;
+}
+
+/* ---------------------------------------------------------------------------------
+ * Counter-based draws for sampled recovery.  The draw of entry (unit, t, j), unit = b * Hkv + h, is a
+ * pure function of the key; both uniforms are 24-bit and lie strictly inside (0, 1).
+ *   c  = (unit << 40) ^ (t << 8) ^ j          64-bit counter
+ *   z  = c + seed * 0x9E3779B97F4A7C15;  z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9;
+ *   z  = (z ^ z >> 27) * 0x94D049BB133111EB;  z ^= z >> 31           (the splitmix64 finaliser)
+ *   u1 = ((z >> 40) + 0.5) / 2^24,   u2 = (((z >> 16) & 0xFFFFFF) + 0.5) / 2^24
+ * --------------------------------------------------------------------------------- */
+void oracle_draw_uniforms(uint32_t seed, int64_t unit, int64_t t, int j, double *u1, double *u2)
+{
+    uint64_t z = ((uint64_t)unit << 40) ^ ((uint64_t)t << 8) ^ (uint64_t)j;
+    z += (uint64_t)seed * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    *u1 = ((double)(z >> 40) + 0.5) / 16777216.0;
+    *u2 = ((double)((z >> 16) & 0xFFFFFFull) + 0.5) / 16777216.0;
+}
+
+/* sampled saliency of one pruned entry: mode 1 Gaussian N(mu, sigma^2) by Box-Muller, mode 2 Exponential
+ * with mean mu (rate 1 / mu) by inversion */
+double oracle_sample_saliency(int mode, double mu, double sigma, double u1, double u2)
+{
+    if (mode == 1) return mu + sigma * sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925286766559 * u2);
+    return -mu * log(u1);
+}
+
+/* ---------------------------------------------------------------------------------
+ * Decode attention with SAMPLED recovery (Sec. "Channel Recovery", Gaussian / Exponential).
+ *   K~[t][j] = K[t][j] if kept, else sample(mode, mu_all[t], sigma_all[t]; seed, unit, t, j) / a[j]
+ * then the attention of oracle_decode_attn (path 0).  recovered (optional): [B][Hkv][S_max][D] double, the
+ * sampled saliencies (0 on kept channels), for distribution checks.
+ * --------------------------------------------------------------------------------- */
+int oracle_decode_attn_sampled(const void *q, const void *k, const void *v, int dtype,
+                               int B, int Hq, int Hkv, int D,
+                               int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                               const int32_t *lens, int S_max,
+                               const uint32_t *mask, const float *mu_all, const float *sigma_all,
+                               const float *a, double scale, int mode, uint32_t seed,
+                               float *out, float *lse, double *recovered)
+{
+    if (!q || !k || !v || !lens || !mask || !mu_all || !a || !out || Hkv <= 0 || Hq % Hkv) return 1;
+    if (mode != 1 && mode != 2) return 1;
+    if (mode == 1 && !sigma_all) return 1;
+    const int G = Hq / Hkv, MW = (D + 31) / 32;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)D);
+    int err = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < Hq; ++i) {
+            const int h = i / G, S = lens[b];
+            float *o = out + ((int64_t)b * Hq + i) * D;
+            for (int c = 0; c < D; ++c) o[c] = 0.f;
+            if (lse) lse[(int64_t)b * Hq + i] = -INFINITY;
+            if (S <= 0) continue;
+            double *s = (double *)malloc(sizeof(double) * (size_t)S);
+            double *acc = (double *)calloc((size_t)D, sizeof(double));
+            if (!s || !acc) { err = 2; free(s); free(acc); continue; }
+            const int64_t unit = (int64_t)b * Hkv + h;
+            const float *au = a + unit * D;
+            const int64_t qb = ((int64_t)b * Hq + i) * D;
+            for (int t = 0; t < S; ++t) {
+                const int64_t u = unit * S_max + t;
+                const int64_t kb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                const uint32_t *m = mask + u * MW;
+                double dot = 0.0;
+                for (int j = 0; j < D; ++j) {
+                    double kt;
+                    if ((m[j / 32] >> (j % 32)) & 1u) {
+                        kt = load_elem(k, kb + j, dtype);
+                    } else {
+                        double u1, u2;
+                        oracle_draw_uniforms(seed, unit, t, j, &u1, &u2);
+                        const double w = oracle_sample_saliency(mode, (double)mu_all[u],
+                                                                sigma_all ? (double)sigma_all[u] : 0.0, u1, u2);
+                        if (recovered && i == h * G) recovered[u * D + j] = w;
+                        kt = w / (double)au[j];
+                    }
+                    dot += load_elem(q, qb + j, dtype) * kt;
+                }
+                s[t] = scale * dot;
+            }
+            double mx = s[0];
+            for (int t = 1; t < S; ++t) if (s[t] > mx) mx = s[t];
+            double den = 0.0;
+            for (int t = 0; t < S; ++t) den += exp(s[t] - mx);
+            for (int t = 0; t < S; ++t) {
+                const double p = exp(s[t] - mx) / den;
+                const int64_t vb = (int64_t)b * stride_b + (int64_t)h * stride_h + (int64_t)t * stride_t;
+                for (int c = 0; c < D; ++c) acc[c] += p * load_elem(v, vb + c, dtype);
+            }
+            for (int c = 0; c < D; ++c) o[c] = (float)acc[c];
+            if (lse) lse[(int64_t)b * Hq + i] = (float)(mx + log(den));
+            free(s); free(acc);
         }
     return err;
 }
