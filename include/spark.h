@@ -78,7 +78,36 @@ typedef struct {
     int64_t n_pool_pages;   /* pages in the pool; every block-table entry must be below it    */
     int32_t flags;          /* bit set of spark_flags (0: none)                               */
     int32_t keep_v;         /* T_v, kept value channels per token; 0 or D: values stay dense   */
+    int32_t select;         /* spark_select: how the kept key channels of a token are chosen  */
+    float   top_p;          /* SPARK_SELECT_TOP_P: share of a token's total saliency to keep   */
+    int32_t n_groups;       /* SPARK_SELECT_GROUPS: rank groups, 1..8                         */
+    float   group_prune[8]; /* SPARK_SELECT_GROUPS: pruning ratio per group, most salient first */
+    int32_t recovery;       /* spark_recovery: distribution that restores the pruned entries   */
+    uint32_t seed;          /* sampled recovery: seed of the per-entry draws                   */
 } spark_params;
+
+/* spark_params.select -- the ratio-free variants of Sec. "Ablation Studies" ("Adaptive Variants").
+ * In every mode `keep` is the capacity of a token's slot list in the page: the number of kept channels
+ * under SPARK_SELECT_FIXED, an upper bound under the two others.
+ *   SPARK_SELECT_TOP_P   (SparK-p) per token, rank the channels by saliency and keep the fewest, at least
+ *                        one and at most `keep`, whose saliencies add up to top_p times the token's total
+ *                        (sums in double, most salient first).
+ *   SPARK_SELECT_GROUPS  (SparK-g) per token, cut the saliency ranks into n_groups segments of D / n_groups
+ *                        ranks (the first D % n_groups segments get one more); segment i keeps its
+ *                        floor((1 - group_prune[i]) * size_i) most salient channels.  `keep` must be at
+ *                        least their sum (spark_group_keep).  The paper lists the ratios and the group
+ *                        counts but not how the groups are formed; ranks per token is this library's reading. */
+typedef enum { SPARK_SELECT_FIXED = 0, SPARK_SELECT_TOP_P = 1, SPARK_SELECT_GROUPS = 2 } spark_select;
+
+/* spark_params.recovery -- the recovery distributions of Sec. "Channel Recovery".  The sampled ones use the
+ * all-channel mean and population deviation of a token's saliencies (App. "Caching Pruned Channel
+ * Statistics"), which the page then carries per token (8 more bytes).  One draw per pruned entry, a pure
+ * function of (seed, sequence, KV head, token, channel): the recovered keys are fixed for the life of the
+ * cache.  Sampled recovery needs dense value rows (keep_v == 0).
+ *   SPARK_RECOVER_DEGENERATE   w~ = mu_pruned (the default everywhere in the paper)
+ *   SPARK_RECOVER_GAUSSIAN     w~ ~ N(mu, sigma^2), not clamped
+ *   SPARK_RECOVER_EXPONENTIAL  w~ ~ Exp(1 / mu), i.e. mean mu */
+typedef enum { SPARK_RECOVER_DEGENERATE = 0, SPARK_RECOVER_GAUSSIAN = 1, SPARK_RECOVER_EXPONENTIAL = 2 } spark_recovery;
 
 /* spark_params.flags */
 typedef enum {
@@ -94,6 +123,10 @@ typedef enum {
 /* T = floor((1 - ratio) * head_dim): the paper's kept-channel count (Sec. "Problem
  * Formulation", below Eq. (cal)).  Host only.  Returns -1 for ratio outside [0, 1). */
 int32_t spark_keep_count(int32_t head_dim, double ratio);
+
+/* Kept channels per token under SPARK_SELECT_GROUPS: sum over the groups of floor((1 - prune[i]) * size_i).
+ * Host only.  -1 on bad arguments. */
+int32_t spark_group_keep(int32_t head_dim, int32_t n_groups, const float *group_prune);
 
 /* Bytes of one page for these parameters (uses head_dim, keep, page_tokens, dtype).
  * Host only.  0 on unsupported parameters. */
@@ -264,6 +297,15 @@ spark_status spark_unpack_pages(const spark_params *p, const void *pages,
                                 const int32_t *packed_lens, int32_t max_tokens,
                                 uint32_t *mask, float *mu, void *vals, void *v,
                                 spark_stream_t stream);
+
+/* spark_unpack_stats -- the all-channel saliency statistics a page carries under a sampled recovery
+ * distribution (App. "Caching Pruned Channel Statistics": mean mu_i and population deviation sigma_i).
+ *   mu_all, sigma_all  OUT [B][Hkv][max_tokens] fp32, zeros for rows t >= packed_lens[b]; either may be NULL.
+ * SPARK_ERR_UNSUPPORTED when recovery is SPARK_RECOVER_DEGENERATE (the page has no such section). */
+spark_status spark_unpack_stats(const spark_params *p, const void *pages,
+                                const int32_t *block_table, int32_t max_blocks,
+                                const int32_t *packed_lens, int32_t max_tokens,
+                                float *mu_all, float *sigma_all, spark_stream_t stream);
 
 /* spark_unpack_value_masks -- the per-token value-channel masks (App. "Pruning Value Cache Channels").
  *   vmask  OUT [B][Hkv][max_tokens][4] uint32, bit (j % 32) of word (j / 32) <=> value channel j kept;

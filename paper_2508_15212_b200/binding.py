@@ -23,7 +23,7 @@ _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
            "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_host", "spark_decode_attn_noalloc", "spark_unpack_pages",
-           "spark_unpack_value_masks", "spark_read_status"]
+           "spark_unpack_value_masks", "spark_unpack_stats", "spark_group_keep", "spark_read_status"]
 
 
 class SparkError(RuntimeError):
@@ -38,10 +38,14 @@ class spark_params(ctypes.Structure):
                 ("page_tokens", ctypes.c_int32), ("dtype", ctypes.c_int32), ("token_budget", ctypes.c_int32),
                 ("pool_kernel", ctypes.c_int32), ("qnorm_eps", ctypes.c_float),
                 ("softmax_scale", ctypes.c_float), ("n_pool_pages", ctypes.c_int64),
-                ("flags", ctypes.c_int32), ("keep_v", ctypes.c_int32)]
+                ("flags", ctypes.c_int32), ("keep_v", ctypes.c_int32),
+                ("select", ctypes.c_int32), ("top_p", ctypes.c_float), ("n_groups", ctypes.c_int32),
+                ("group_prune", ctypes.c_float * 8), ("recovery", ctypes.c_int32), ("seed", ctypes.c_uint32)]
 
 
 SPARK_FLAG_OVERLAP_PREVIOUS = 1
+SPARK_SELECT_FIXED, SPARK_SELECT_TOP_P, SPARK_SELECT_GROUPS = 0, 1, 2
+SPARK_RECOVER_DEGENERATE, SPARK_RECOVER_GAUSSIAN, SPARK_RECOVER_EXPONENTIAL = 0, 1, 2
 
 
 _lib = None
@@ -82,6 +86,10 @@ def lib() -> ctypes.CDLL:
         L.spark_unpack_pages.argtypes = [P, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp]
         L.spark_unpack_value_masks.restype = i32
         L.spark_unpack_value_masks.argtypes = [P, vp, vp, i32, vp, i32, vp, vp]
+        L.spark_unpack_stats.restype = i32
+        L.spark_unpack_stats.argtypes = [P, vp, vp, i32, vp, i32, vp, vp, vp]
+        L.spark_group_keep.restype = i32
+        L.spark_group_keep.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_float)]
         L.spark_read_status.restype = i32
         L.spark_read_status.argtypes = [vp, vp]
         _lib = L
@@ -111,10 +119,18 @@ def _stream():
 
 def make_params(*, batch, n_q_heads, n_kv_heads, window, keep, dtype, n_pool_pages, head_dim=128,
                 page_tokens=16, token_budget=0, pool_kernel=7, qnorm_eps=0.0, softmax_scale=0.0,
-                flags=0, keep_v=0) -> spark_params:
+                flags=0, keep_v=0, top_p=None, group_prune=None, recovery=0, seed=0) -> spark_params:
+    """A parameter block.  `top_p` selects SparK-p, `group_prune` (ratios, most salient rank group first)
+    selects SparK-g; `keep` is then the capacity of a token's slot list."""
     code = dtype if isinstance(dtype, int) else _DTYPE_CODE[dtype]
+    assert top_p is None or group_prune is None
+    select = SPARK_SELECT_TOP_P if top_p is not None else (SPARK_SELECT_GROUPS if group_prune is not None else SPARK_SELECT_FIXED)
+    ratios = list(group_prune) if group_prune is not None else []
+    assert len(ratios) <= 8
+    arr = (ctypes.c_float * 8)(*(ratios + [0.0] * (8 - len(ratios))))
     return spark_params(batch, n_q_heads, n_kv_heads, head_dim, window, keep, page_tokens, code,
-                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages, flags, keep_v)
+                        token_budget, pool_kernel, qnorm_eps, softmax_scale, n_pool_pages, flags, keep_v,
+                        select, float(top_p) if top_p is not None else 0.0, len(ratios), arr, int(recovery), int(seed))
 
 
 # ---- host-only helpers -----------------------------------------------------------------------------
@@ -128,6 +144,12 @@ def spark_last_launch_count() -> int:
 
 def spark_keep_count(head_dim: int, ratio: float) -> int:
     return int(lib().spark_keep_count(head_dim, ratio))
+
+
+def spark_group_keep(head_dim: int, group_prune) -> int:
+    ratios = list(group_prune)
+    arr = (ctypes.c_float * len(ratios))(*ratios)
+    return int(lib().spark_group_keep(head_dim, len(ratios), arr))
 
 
 def spark_page_bytes(p: spark_params) -> int:
@@ -247,6 +269,13 @@ def spark_unpack_value_masks(p: spark_params, pages, block_table, packed_lens, m
     _check(lib().spark_unpack_value_masks(ctypes.byref(p), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
                                           _ptr(packed_lens), int(max_tokens), _ptr(vmask), _stream()),
            "spark_unpack_value_masks")
+
+
+def spark_unpack_stats(p: spark_params, pages, block_table, packed_lens, max_tokens, mu_all, sigma_all,
+                       max_blocks=None) -> None:
+    _check(lib().spark_unpack_stats(ctypes.byref(p), _ptr(pages), _ptr(block_table), _blocks(block_table, max_blocks),
+                                    _ptr(packed_lens), int(max_tokens), _ptr(mu_all), _ptr(sigma_all), _stream()),
+           "spark_unpack_stats")
 
 
 def spark_read_status(workspace: torch.Tensor) -> int:

@@ -24,7 +24,8 @@ class SparkCache:
                  max_tokens: int, device="cuda", block_table: Optional[torch.Tensor] = None,
                  n_pool_pages: Optional[int] = None, token_budget: int = 0, pool_kernel: int = 7,
                  softmax_scale: float = 0.0, pages: Optional[torch.Tensor] = None, flags: int = 0,
-                 keep_v: int = 0, guard: bool = False):
+                 keep_v: int = 0, guard: bool = False, top_p: Optional[float] = None, group_prune=None,
+                 recovery: int = 0, seed: int = 0):
         self.device = torch.device(device)
         self.guard = bool(guard)          # debugging aid: canary bands around every buffer the library writes
         self._bands = []                  # (name, raw uint8 tensor, payload bytes)
@@ -46,7 +47,8 @@ class SparkCache:
         self.params = B.make_params(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window,
                                     keep=keep, dtype=_TDT[dtype], n_pool_pages=n_pool_pages,
                                     token_budget=token_budget, pool_kernel=pool_kernel,
-                                    softmax_scale=softmax_scale, flags=flags, keep_v=keep_v)
+                                    softmax_scale=softmax_scale, flags=flags, keep_v=keep_v, top_p=top_p,
+                                    group_prune=group_prune, recovery=recovery, seed=seed)
         self.page_bytes = B.spark_page_bytes(self.params)
         assert self.page_bytes > 0
         self.pages = pages if pages is not None else self._alloc("pages", n_pool_pages * self.page_bytes, zero=True)
@@ -124,7 +126,7 @@ class SparkCache:
                                  max_blocks=self.table_blocks, stream=stream)
 
     # -- inspection ------------------------------------------------------------------------------
-    def unpack(self, want_vals=True, want_v=True, want_vmask=False) -> Dict[str, torch.Tensor]:
+    def unpack(self, want_vals=True, want_v=True, want_vmask=False, want_stats=False) -> Dict[str, torch.Tensor]:
         p, n = self.params, self.max_tokens
         tdt = _TDT[self.dtype]
         out = dict(mask=torch.empty(p.batch, p.n_kv_heads, n, 4, dtype=torch.int32, device=self.device),
@@ -139,6 +141,11 @@ class SparkCache:
             out["vmask"] = torch.empty(p.batch, p.n_kv_heads, n, 4, dtype=torch.int32, device=self.device)
             B.spark_unpack_value_masks(p, self.pages, self.block_table, self.packed_lens, n, out["vmask"],
                                        max_blocks=self.table_blocks)
+        if want_stats:
+            out["mu_all"] = torch.empty(p.batch, p.n_kv_heads, n, dtype=torch.float32, device=self.device)
+            out["sigma_all"] = torch.empty(p.batch, p.n_kv_heads, n, dtype=torch.float32, device=self.device)
+            B.spark_unpack_stats(p, self.pages, self.block_table, self.packed_lens, n, out["mu_all"], out["sigma_all"],
+                                 max_blocks=self.table_blocks)
         return out
 
     def status(self) -> int:

@@ -32,7 +32,29 @@ spark_status spark::check_params(const spark_params* p)
     if (!(p->qnorm_eps >= 0.f) || !(p->softmax_scale >= 0.f)) return SPARK_ERR_BAD_SHAPE;
     if (p->flags & ~SPARK_FLAG_OVERLAP_PREVIOUS) return SPARK_ERR_BAD_SHAPE;
     if (p->keep_v < 0 || p->keep_v > p->head_dim) return SPARK_ERR_BAD_SHAPE;
+    if (p->select < SPARK_SELECT_FIXED || p->select > SPARK_SELECT_GROUPS) return SPARK_ERR_BAD_SHAPE;
+    if (p->select == SPARK_SELECT_TOP_P && (!(p->top_p > 0.f) || !(p->top_p <= 1.f))) return SPARK_ERR_BAD_SHAPE;
+    if (p->select == SPARK_SELECT_GROUPS) {
+        const int need = group_keep(p->head_dim, p->n_groups, p->group_prune);
+        if (need < 0 || need > p->keep) return SPARK_ERR_BAD_SHAPE;
+    }
+    if (p->recovery < SPARK_RECOVER_DEGENERATE || p->recovery > SPARK_RECOVER_EXPONENTIAL) return SPARK_ERR_BAD_SHAPE;
+    if (p->recovery != SPARK_RECOVER_DEGENERATE && value_keep(p->keep_v) < kHeadDim) return SPARK_ERR_UNSUPPORTED;
     return SPARK_OK;
+}
+
+int spark::group_keep(int head_dim, int n_groups, const float* prune)
+{
+    if (head_dim < 1 || n_groups < 1 || n_groups > 8 || n_groups > head_dim || !prune) return -1;
+    int total = 0;
+    for (int i = 0; i < n_groups; ++i) {
+        if (!(prune[i] >= 0.f) || !(prune[i] <= 1.f)) return -1;
+        const int size = head_dim / n_groups + (i < head_dim % n_groups ? 1 : 0);
+        // the small offset absorbs binary representation error of ratios whose product is an integer
+        int kp = static_cast<int>(floor((1.0 - static_cast<double>(prune[i])) * size + 1e-9));
+        total += kp < 0 ? 0 : (kp > size ? size : kp);
+    }
+    return total;
 }
 
 extern "C" {
@@ -48,13 +70,19 @@ int32_t spark_keep_count(int32_t head_dim, double ratio)
     return static_cast<int32_t>(floor((1.0 - ratio) * head_dim + 1e-9));
 }
 
+int32_t spark_group_keep(int32_t head_dim, int32_t n_groups, const float* group_prune)
+{
+    return group_keep(head_dim, n_groups, group_prune);
+}
+
 size_t spark_page_bytes(const spark_params* p)
 {
     if (!p || p->head_dim != kHeadDim || p->page_tokens != kPageTokens) return 0;
     if (p->dtype != SPARK_F32 && p->dtype != SPARK_BF16) return 0;
     if (p->keep < 1 || p->keep > kHeadDim) return 0;
     if (p->keep_v < 0 || p->keep_v > kHeadDim) return 0;
-    return static_cast<size_t>(make_layout(p->dtype, p->keep, p->keep_v).page_bytes);
+    if (p->recovery < SPARK_RECOVER_DEGENERATE || p->recovery > SPARK_RECOVER_EXPONENTIAL) return 0;
+    return static_cast<size_t>(make_layout(*p).page_bytes);
 }
 
 size_t spark_algorithmic_bytes_per_token(const spark_params* p)
@@ -62,7 +90,8 @@ size_t spark_algorithmic_bytes_per_token(const spark_params* p)
     if (!p || p->keep < 1 || p->keep > p->head_dim || p->keep_v < 0 || p->keep_v > p->head_dim) return 0;
     const size_t e = (p->dtype == SPARK_BF16) ? 2 : 4;
     const int tv = value_keep(p->keep_v);
-    return e * p->keep + 16 + 4 + (tv < kHeadDim ? e * tv + 16 : e * p->head_dim);
+    const size_t stats = (p->recovery != SPARK_RECOVER_DEGENERATE) ? 8 : 0;       // all-channel mean and deviation
+    return e * p->keep + 16 + 4 + stats + (tv < kHeadDim ? e * tv + 16 : e * p->head_dim);
 }
 
 spark_status spark_workspace_bytes(const spark_params* p, int64_t max_seq_tokens,
@@ -204,7 +233,23 @@ spark_status spark_unpack_pages(const spark_params* p, const void* pages, const 
     if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
         return SPARK_ERR_BAD_SHAPE;
     return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, mask, mu, vals, v, nullptr,
-                         static_cast<cudaStream_t>(stream));
+                         nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+spark_status spark_unpack_stats(const spark_params* p, const void* pages, const int32_t* block_table,
+                                int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
+                                float* mu_all, float* sigma_all, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!pages || !packed_lens) return SPARK_ERR_NULL;
+    if (p->recovery == SPARK_RECOVER_DEGENERATE) return SPARK_ERR_UNSUPPORTED;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
+    if (max_tokens < 0 || max_blocks < 0 || max_blocks > kMaxBlocksArg) return SPARK_ERR_BAD_SHAPE;
+    if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
+        return SPARK_ERR_BAD_SHAPE;
+    return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, nullptr, nullptr, nullptr,
+                         nullptr, nullptr, mu_all, sigma_all, static_cast<cudaStream_t>(stream));
 }
 
 spark_status spark_unpack_value_masks(const spark_params* p, const void* pages, const int32_t* block_table,
@@ -219,7 +264,7 @@ spark_status spark_unpack_value_masks(const spark_params* p, const void* pages, 
     if ((static_cast<int64_t>(max_tokens) + kPageTokens - 1) / kPageTokens > max_blocks)
         return SPARK_ERR_BAD_SHAPE;
     return launch_unpack(*p, pages, block_table, max_blocks, packed_lens, max_tokens, nullptr, nullptr, nullptr,
-                         nullptr, vmask, static_cast<cudaStream_t>(stream));
+                         nullptr, vmask, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 spark_status spark_read_status(const void* workspace, spark_stream_t stream)

@@ -26,6 +26,7 @@ constexpr int kWorkspaceHeader = 256;
 //          fragment reads together fall into eight different 4-byte banks.
 //   mask : [16][4] uint32, bit (j % 32) of word (j / 32) set <=> channel j kept
 //   mu   : [16] float, mean saliency of the pruned channels
+//   stats: (sampled recovery only) [16] float mean and [16] float population deviation of ALL the token's saliencies
 //   v    : dense values (keep_v == 128): [16][128] elements, the value rows.  In bf16 pages the 16-byte
 //          chunks of row p are stored at chunk index (c ^ (p & 7)), which makes the transposing matrix
 //          loads of the decode kernel free of bank conflicts; fp32 pages store rows plainly.
@@ -38,6 +39,8 @@ struct PageLayout {
     int keep_v;      // T_v (128: dense value rows)
     int mask_off;
     int mu_off;
+    int stats_off;   // [16] float all-channel mean, [16] float population deviation (sampled recovery only)
+    int recovery;    // spark_recovery
     int v_off;
     int vmask_off;   // meaningful when keep_v < 128
     int page_bytes;
@@ -46,7 +49,7 @@ struct PageLayout {
 // spark_params.keep_v -> T_v (0 and 128 both mean dense value rows)
 __host__ __device__ inline int value_keep(int keep_v) { return (keep_v <= 0 || keep_v >= kHeadDim) ? kHeadDim : keep_v; }
 
-__host__ __device__ inline PageLayout make_layout(int dtype, int keep, int keep_v)
+__host__ __device__ inline PageLayout make_layout(int dtype, int keep, int keep_v, int recovery)
 {
     PageLayout L;
     L.esize = (dtype == SPARK_BF16) ? 2 : 4;
@@ -54,7 +57,9 @@ __host__ __device__ inline PageLayout make_layout(int dtype, int keep, int keep_
     L.keep_v = value_keep(keep_v);
     L.mask_off = keep * kPageTokens * L.esize;
     L.mu_off = L.mask_off + kPageTokens * 16;
-    L.v_off = L.mu_off + kPageTokens * 4;
+    L.stats_off = L.mu_off + kPageTokens * 4;
+    L.recovery = recovery;
+    L.v_off = L.stats_off + (recovery != SPARK_RECOVER_DEGENERATE ? 2 * kPageTokens * 4 : 0);
     L.vmask_off = L.v_off + L.keep_v * kPageTokens * L.esize;
     L.page_bytes = L.vmask_off + (L.keep_v < kHeadDim ? kPageTokens * 16 : 0);
     return L;
@@ -108,7 +113,10 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
 
 spark_status launch_unpack(const spark_params& p, const void* pages, const int32_t* block_table,
                            int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
-                           uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, cudaStream_t stream);
+                           uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, float* mu_all,
+                           float* sigma_all, cudaStream_t stream);
+inline PageLayout make_layout(const spark_params& p) { return make_layout(p.dtype, p.keep, p.keep_v, p.recovery); }
+int group_keep(int head_dim, int n_groups, const float* prune);
 
 spark_status launch_decode(const spark_params& p, const void* q, const void* pages,
                            const int32_t* block_table, int32_t max_blocks, const int32_t* packed_lens,

@@ -67,20 +67,18 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 // `mu_off` >= 0 (`inv_pruned` = 1 / (D - T), or 0 when nothing is pruned: the mean is taken as a product
 // in double, which rounds to the same float as the quotient except on a rounding boundary of the double).
 // ------------------------------------------------------------------------------------------------
-template <bool kBf16>
-__device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, int mask_off, int mu_off,
-                                           int p, int T, int lane,
-                                           const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4],
-                                           double inv_pruned = 0.0)
+// How the kept key channels of a token are chosen, and which statistics the page stores.
+struct SelectArgs {
+    int select;                   // spark_select
+    float top_p;                  // SPARK_SELECT_TOP_P
+    unsigned rank_keep[4];        // SPARK_SELECT_GROUPS: bit r set <=> the channel of saliency rank r is kept
+    int recovery;                 // spark_recovery: a sampled distribution needs the all-channel statistics
+};
+
+// Exact top-T of the warp's 128 keys: kept[i] for the lane's four channels (see pack_token).
+__device__ __forceinline__ void select_top_t(const unsigned (&key)[4], int T, int lane, bool (&kept)[4])
 {
     const unsigned lt = (1u << lane) - 1u;
-    float w[4];
-    unsigned key[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
-        key[i] = __float_as_uint(w[i]);
-    }
     // T-th largest key by radix descent over the bits in which the 128 keys differ.  The descent
     // stops as soon as a candidate threshold has exactly T keys at or above it (then those are the
     // kept set and no tie can straddle the boundary); otherwise it ends with the exact T-th largest
@@ -98,7 +96,6 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
         if (cnt >= T) thr = cand;
         if (cnt == T) { exact = true; break; }
     }
-    bool kept[4];
     if (exact) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) kept[i] = key[i] >= thr;
@@ -121,6 +118,118 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
             rank += eq ? 1 : 0;
         }
     }
+}
+
+// The ratio-free selection rules (Sec. "Ablation Studies", adaptive variants) need every channel's saliency
+// RANK, so the warp sorts its 128 keys: a bitonic network over (saliency bits, 127 - channel), descending,
+// four consecutive ranks per lane.  SparK-p then keeps the shortest rank prefix whose saliencies (summed in
+// double, most salient first) reach top_p of the token's total, at least one and at most `cap` channels;
+// SparK-g keeps the ranks listed in rank_keep.  Returns kept[i] for the lane's four CHANNELS and the count.
+__device__ __forceinline__ int select_by_rank(const unsigned (&key)[4], int lane, const SelectArgs& sel, int cap,
+                                              bool (&kept)[4])
+{
+    unsigned long long K[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        K[e] = (static_cast<unsigned long long>(key[e]) << 7) | static_cast<unsigned>(127 - (4 * lane + e));
+#pragma unroll
+    for (int size = 2; size <= 128; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride >= 4) {
+                const bool lower = ((4 * lane) & stride) == 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const unsigned long long other = __shfl_xor_sync(kFullMask, K[e], stride >> 2);
+                    const bool down = ((4 * lane + e) & size) == 0;     // this block ends up descending
+                    const bool take_max = (lower == down);
+                    K[e] = take_max ? (K[e] > other ? K[e] : other) : (K[e] < other ? K[e] : other);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if ((e & stride) == 0) {
+                        const bool down = ((4 * lane + e) & size) == 0;
+                        const unsigned long long x = K[e], y = K[e ^ stride];
+                        const unsigned long long hi = x > y ? x : y, lo = x > y ? y : x;
+                        K[e] = down ? hi : lo;
+                        K[e ^ stride] = down ? lo : hi;
+                    }
+            }
+        }
+    }
+    unsigned rk[4] = {sel.rank_keep[0], sel.rank_keep[1], sel.rank_keep[2], sel.rank_keep[3]};
+    if (sel.select == SPARK_SELECT_TOP_P) {
+        double c[4];
+        double run = 0.0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            run += static_cast<double>(__uint_as_float(static_cast<unsigned>(K[e] >> 7)));
+            c[e] = run;
+        }
+        double incl = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(kFullMask, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const double total = __shfl_sync(kFullMask, incl, 31);
+        const double need = static_cast<double>(sel.top_p) * total;
+        const double before = incl - run;
+        int below = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) below += (before + c[e] < need) ? 1 : 0;
+        int n = __reduce_add_sync(kFullMask, below) + 1;       // first rank whose running sum reaches `need`
+        n = n > kHeadDim ? kHeadDim : n;
+        n = n > cap ? cap : n;
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi)
+            rk[wi] = n >= 32 * (wi + 1) ? 0xffffffffu : (n > 32 * wi ? ((1u << (n - 32 * wi)) - 1u) : 0u);
+    }
+    unsigned m[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int r = 4 * lane + e;
+        if ((rk[r >> 5] >> (r & 31)) & 1u) {
+            const int j = 127 - static_cast<int>(K[e] & 127u);
+#pragma unroll
+            for (int wi = 0; wi < 4; ++wi)
+                if ((j >> 5) == wi) m[wi] |= 1u << (j & 31);
+        }
+    }
+    int n_kept = 0;
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {
+        m[wi] = __reduce_or_sync(kFullMask, m[wi]);
+        n_kept += __popc(m[wi]);
+    }
+    unsigned mine = m[0];
+#pragma unroll
+    for (int wi = 1; wi < 4; ++wi)
+        if ((lane >> 3) == wi) mine = m[wi];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) kept[i] = (mine >> (4 * (lane & 7) + i)) & 1u;
+    return n_kept;
+}
+
+template <bool kBf16>
+__device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, int mask_off, int mu_off,
+                                           int p, int T, int lane,
+                                           const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4],
+                                           double inv_pruned = 0.0, const SelectArgs* sel = nullptr, int stats_off = -1)
+{
+    const unsigned lt = (1u << lane) - 1u;
+    float w[4];
+    unsigned key[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        w[i] = __fmul_rn(a[i], fabsf(kf[i]));                 // the one rounding that decides selection
+        key[i] = __float_as_uint(w[i]);
+    }
+    bool kept[4];
+    int n_kept = T;
+    if (sel && sel->select != SPARK_SELECT_FIXED) n_kept = select_by_rank(key, lane, *sel, T, kept);   // warp-uniform
+    else select_top_t(key, T, lane, kept);
     // slot of each kept channel = kept channels below it
     int slot = 0;
     unsigned nib = 0;
@@ -150,8 +259,29 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
     if (mu_off < 0) return;                                   // warp-uniform
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
-    if (lane == 0)
-        reinterpret_cast<float*>(image + mu_off)[p] = static_cast<float>(pruned * inv_pruned);
+    if (lane == 0) {
+        float mu;
+        if (sel && sel->select != SPARK_SELECT_FIXED)
+            mu = n_kept < kHeadDim ? static_cast<float>(pruned / static_cast<double>(kHeadDim - n_kept)) : 0.f;
+        else
+            mu = static_cast<float>(pruned * inv_pruned);
+        reinterpret_cast<float*>(image + mu_off)[p] = mu;
+    }
+    if (stats_off < 0) return;                                // warp-uniform
+    // all-channel mean and population deviation of the token's saliencies (sampled recovery)
+    double s1 = (static_cast<double>(w[0]) + static_cast<double>(w[1])) + (static_cast<double>(w[2]) + static_cast<double>(w[3]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s1 += __shfl_xor_sync(kFullMask, s1, o);
+    const double mean = s1 / static_cast<double>(kHeadDim);
+    double s2 = 0.0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const double d = static_cast<double>(w[i]) - mean; s2 += d * d; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(kFullMask, s2, o);
+    if (lane == 0) {
+        reinterpret_cast<float*>(image + stats_off)[p] = static_cast<float>(mean);
+        reinterpret_cast<float*>(image + stats_off)[kPageTokens + p] = static_cast<float>(sqrt(s2 / static_cast<double>(kHeadDim)));
+    }
 }
 
 // Key entries and value entries of one token row into the page image.  A lane owns channels 4*lane ..
@@ -160,7 +290,7 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
 template <bool kBf16>
 __device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLayout& L, int p, int lane,
                                               const float (&a)[4], const void* k, const void* v, int64_t row,
-                                              double inv_pruned)
+                                              double inv_pruned, const SelectArgs& sel)
 {
     unsigned kraw[4], vraw[4];
     float kf[4];
@@ -191,7 +321,8 @@ __device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLa
         const float one[4] = {1.f, 1.f, 1.f, 1.f};
         pack_token<kBf16>(image, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
     }
-    pack_token<kBf16>(image, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned);
+    pack_token<kBf16>(image, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned, &sel,
+                      L.recovery != SPARK_RECOVER_DEGENERATE ? L.stats_off : -1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -218,6 +349,7 @@ struct CompressArgs {
     int64_t n_pool_pages;
     PageLayout L;
     double inv_pruned;            // 1 / (D - T), 0 when T = D
+    SelectArgs sel;
     int* status;
 };
 
@@ -246,7 +378,7 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
         const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
                             static_cast<int64_t>(src_t) * A.st + lane * 4;
-        pack_token_kv<kBf16>(image, L, p, lane, a, A.k, A.v, row, A.inv_pruned);
+        pack_token_kv<kBf16>(image, L, p, lane, a, A.k, A.v, row, A.inv_pruned, A.sel);
     }
     __syncthreads();
 
@@ -278,6 +410,7 @@ struct AppendArgs {
     const float* qnorm;
     int32_t* packed_lens;
     double inv_pruned;            // 1 / (D - T), 0 when T = D
+    SelectArgs sel;
     int* status;
 };
 
@@ -307,7 +440,7 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
     const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
     const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
-    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned);
+    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
 }
 
 __global__ void append_advance_kernel(AppendArgs A)
@@ -318,6 +451,24 @@ __global__ void append_advance_kernel(AppendArgs A)
     if (t >= 0 && t / kPageTokens < A.max_blocks) A.packed_lens[b] = t + 1;
 }
 
+// selection arguments of a parameter block (the rank mask of SparK-g is laid out on the host)
+static SelectArgs make_select(const spark_params& p)
+{
+    SelectArgs s;
+    s.select = p.select; s.top_p = p.top_p; s.recovery = p.recovery;
+    s.rank_keep[0] = s.rank_keep[1] = s.rank_keep[2] = s.rank_keep[3] = 0u;
+    if (p.select == SPARK_SELECT_GROUPS) {
+        int start = 0;
+        for (int i = 0; i < p.n_groups; ++i) {
+            const int size = kHeadDim / p.n_groups + (i < kHeadDim % p.n_groups ? 1 : 0);
+            const int kp = group_keep(size, 1, &p.group_prune[i]);          // floor((1 - prune) * size)
+            for (int r = start; r < start + kp; ++r) s.rank_keep[r >> 5] |= 1u << (r & 31);
+            start += size;
+        }
+    }
+    return s;
+}
+
 spark_status launch_append(const spark_params& p, const void* k_new, const void* v_new, void* pages,
                            const int32_t* block_table, int32_t max_blocks, const float* qnorm,
                            int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches)
@@ -325,8 +476,9 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     AppendArgs A;
     A.k_new = k_new; A.v_new = v_new; A.pages = static_cast<unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.B = p.batch; A.Hkv = p.n_kv_heads; A.keep = p.keep; A.n_pool_pages = p.n_pool_pages;
-    A.L = make_layout(p.dtype, p.keep, p.keep_v); A.qnorm = qnorm; A.packed_lens = packed_lens;
+    A.L = make_layout(p); A.qnorm = qnorm; A.packed_lens = packed_lens;
     A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
+    A.sel = make_select(p);
     A.status = static_cast<int*>(workspace);
     const dim3 grid(p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16) append_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(A);
@@ -353,6 +505,8 @@ struct UnpackArgs {
     void* vals;
     void* v;
     uint32_t* vmask;
+    float* mu_all;
+    float* sigma_all;
 };
 
 __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
@@ -381,6 +535,14 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
         for (int p = threadIdx.x; p < kPageTokens; p += blockDim.x) {
             if (t0 + p >= A.max_tokens) continue;
             A.mu[row0 + p] = (page && t0 + p < len) ? reinterpret_cast<const float*>(page + L.mu_off)[p] : 0.f;
+        }
+    if (A.mu_all || A.sigma_all)                                  // only called for layouts that carry the section
+        for (int p = threadIdx.x; p < kPageTokens; p += blockDim.x) {
+            if (t0 + p >= A.max_tokens) continue;
+            const bool live = page && t0 + p < len;
+            const float* st = reinterpret_cast<const float*>(page + L.stats_off);
+            if (A.mu_all) A.mu_all[row0 + p] = live ? st[p] : 0.f;
+            if (A.sigma_all) A.sigma_all[row0 + p] = live ? st[kPageTokens + p] : 0.f;
         }
     if (A.vals)
         for (int i = threadIdx.x; i < kPageTokens * T; i += blockDim.x) {
@@ -467,8 +629,9 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
     A.lens = packed_lens; A.gather = evict ? kept_tokens : nullptr; A.gather_stride = evict ? p.token_budget : 0;
     A.qnorm = qnorm; A.pages = static_cast<unsigned char*>(pages);
     A.block_table = block_table; A.max_blocks = max_blocks; A.Hkv = p.n_kv_heads; A.keep = p.keep;
-    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep, p.keep_v); A.status = status;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p); A.status = status;
     A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
+    A.sel = make_select(p);
     const dim3 grid(n_blocks, p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16)
         compress_pages_kernel<__nv_bfloat16><<<grid, 256, A.L.page_bytes, stream>>>(A);
@@ -481,15 +644,16 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
 
 spark_status launch_unpack(const spark_params& p, const void* pages, const int32_t* block_table,
                            int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
-                           uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, cudaStream_t stream)
+                           uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, float* mu_all,
+                           float* sigma_all, cudaStream_t stream)
 {
     const int n_blocks = (max_tokens + kPageTokens - 1) / kPageTokens;
     if (n_blocks == 0) return SPARK_OK;
     UnpackArgs A;
     A.pages = static_cast<const unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.lens = packed_lens; A.max_tokens = max_tokens; A.Hkv = p.n_kv_heads;
-    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p.dtype, p.keep, p.keep_v);
-    A.mask = mask; A.mu = mu; A.vals = vals; A.v = v; A.vmask = vmask;
+    A.n_pool_pages = p.n_pool_pages; A.L = make_layout(p);
+    A.mask = mask; A.mu = mu; A.vals = vals; A.v = v; A.vmask = vmask; A.mu_all = mu_all; A.sigma_all = sigma_all;
     unpack_pages_kernel<<<dim3(n_blocks, p.n_kv_heads, p.batch), 128, 0, stream>>>(A);
     if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
     return SPARK_OK;

@@ -1,14 +1,24 @@
-// Decode attention over the packed SparK cache, fp32 storage (Sec. "Channel Recovery", degenerate
-// distribution, then the softmax attention of Sec. "Preliminaries"), and the dispatch of
-// spark_decode_attn to the per-dtype kernels.
+// Decode attention over the packed SparK cache on the CUDA cores: fp32 storage with the degenerate recovery
+// distribution, and either storage type with a SAMPLED recovery distribution (Sec. "Channel Recovery":
+// Gaussian / Exponential; then the softmax attention of Sec. "Preliminaries"); also the dispatch of
+// spark_decode_attn to the kernels.
 //
 // With a[j] = max(|q-bar_j|, eps) the reconstructed key is K~[t][j] = K[t][j] on kept channels and
 // mu[t] / a[j] on pruned ones, so for one query head
 //     q . K~[t] = sum_{j kept} q[j] * (K[t][j] - mu[t] / a[j])  +  mu[t] * sum_j q[j] / a[j].
 // This kernel evaluates that form with fp32 FMAs: a lane owns a token for the scores (it walks the set
 // bits of the token's mask and gathers the query entries from a shared table) and four channels for
-// P.V.  fp32 caches are the small high-precision configuration; the bf16 kernel carries the
+// P.V.  fp32 caches are the small high-precision configuration; the bf16 tensor-core kernel carries the
 // bandwidth-bound workloads.
+//
+// Sampled recovery (template parameter R = 1 Gaussian, 2 Exponential): every pruned entry of a token is a
+// draw w~ from the distribution built on the token's all-channel statistics (mean, population deviation;
+// App. "Caching Pruned Channel Statistics", stored per token in the page), and the recovered key is
+// w~ / a[j].  The draw is a pure function of (seed, unit, token, channel) -- the splitmix64 mixer of a
+// 64-bit counter, two 24-bit uniforms, Box-Muller or inversion -- so the recovered keys never change while
+// the cache lives.  The algebraic folding of the degenerate rule does not apply: the lane walks all 128
+// channels of its token, which makes this the method's slow variant (the paper's ablation also ranks it
+// below the degenerate rule).
 #include "spark_decode_common.cuh"
 
 namespace spark {
@@ -17,6 +27,30 @@ constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kDecodeThreads = kConsumerThreads + 32;     // + producer warp
 constexpr int kStepTokens = 2 * kPageTokens;              // a lane per token: two pages per step
+
+// one sampled saliency: Gaussian N(mu, sigma^2) by Box-Muller (R = 1) or Exponential with mean mu by
+// inversion (R = 2), from the counter (unit, t, j)
+template <int R>
+__device__ __forceinline__ float sample_saliency(unsigned seed, unsigned long long unit_t, int j, float mu, float sigma)
+{
+    unsigned long long z = unit_t ^ static_cast<unsigned long long>(j);
+    z += static_cast<unsigned long long>(seed) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    // (x + 0.5) / 2^24 with x < 2^24: the sum needs 25 bits, so it is formed in double and rounded once
+    const float u1 = static_cast<float>((static_cast<double>(z >> 40) + 0.5) * (1.0 / 16777216.0));
+    if (R == 2) return -mu * logf(u1);
+    const float u2 = static_cast<float>((static_cast<double>((z >> 16) & 0xFFFFFFull) + 0.5) * (1.0 / 16777216.0));
+    return fmaf(sigma * sqrtf(-2.0f * logf(u1)), cospif(2.0f * u2), mu);
+}
+
+template <typename E> __device__ __forceinline__ float load_query(const void* q, int64_t i);
+template <> __device__ __forceinline__ float load_query<float>(const void* q, int64_t i) { return static_cast<const float*>(q)[i]; }
+template <> __device__ __forceinline__ float load_query<__nv_bfloat16>(const void* q, int64_t i)
+{
+    return bf16_bits_to_float(static_cast<const unsigned short*>(q)[i]);
+}
 
 template <int G> struct SmemF32 {
     static constexpr int GP = ((G + 1 + 3) / 4) * 4;     // floats per table entry: G scaled queries + 1/a
@@ -28,9 +62,11 @@ template <int G> struct SmemF32 {
     static constexpr int kFixed = (kMerge + merge_bytes(kConsumerWarps, G) + 127) / 128 * 128;   // prefix and ring start here
 };
 
-template <int G>
-__global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const DecodeArgs A)
+template <int G, typename E, int R>
+__global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const DecodeArgs A)
 {
+    constexpr bool kBf16 = (sizeof(E) == 2);
+    static_assert(!(kBf16 && R == 0), "bf16 storage with the degenerate rule runs on the tensor-core kernel");
     using S = SmemF32<G>;
     constexpr int GP = S::GP, GPP = S::GPP;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -74,8 +110,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
             const int j = idx / GP, e = idx - j * GP;
             float val = 0.f;
             if (e < G)
-                val = static_cast<const float*>(A.q)[(static_cast<int64_t>(b) * A.Hq + h * G + e) * kHeadDim + j] *
-                      A.scale_log2e;
+                val = load_query<E>(A.q, (static_cast<int64_t>(b) * A.Hq + h * G + e) * kHeadDim + j) * A.scale_log2e;
             else if (e == G)
                 val = 1.0f / A.qnorm[(static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + j];
             qtab[idx] = val;
@@ -119,35 +154,75 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                     const unsigned char* page = sbase + (lane >> 4) * L.page_bytes;
                     const int p = lane & 15;
                     const uint4 mk = *reinterpret_cast<const uint4*>(page + L.mask_off + p * 16);
-                    const float mu = *reinterpret_cast<const float*>(page + L.mu_off + p * 4);
                     const unsigned words[4] = {mk.x, mk.y, mk.z, mk.w};
-                    const float* vp = reinterpret_cast<const float*>(page) + p;     // slot s at vp[16 s]
+                    // kept slot s of token p (see val_offset): fp32 rows hold token p at element p, bf16 rows at
+                    // element (p & 7) * 2 + (p >> 3); rows are 16 elements apart
+                    const unsigned char* vp = page + (kBf16 ? ((p & 7) * 2 + (p >> 3)) * 2 : p * 4);
+                    constexpr int kRowBytes = kPageTokens * static_cast<int>(sizeof(E));
                     float a[G];
 #pragma unroll
                     for (int gg = 0; gg < G; ++gg) a[gg] = 0.f;
+                    if (R == 0) {
+                        const float mu = *reinterpret_cast<const float*>(page + L.mu_off + p * 4);
 #pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) {
-                        unsigned w = words[wi];
-                        const float* tb = qtab + wi * 32 * GP;
-                        while (w) {
-                            const int bp = __ffs(w) - 1;
-                            w &= w - 1;
-                            const float* e = tb + bp * GP;
-                            const float kv = *vp;
-                            vp += kPageTokens;
-                            float tv[GP];
+                        for (int wi = 0; wi < 4; ++wi) {
+                            unsigned w = words[wi];
+                            const float* tb = qtab + wi * 32 * GP;
+                            while (w) {
+                                const int bp = __ffs(w) - 1;
+                                w &= w - 1;
+                                const float* e = tb + bp * GP;
+                                const float kv = *reinterpret_cast<const float*>(vp);
+                                vp += kRowBytes;
+                                float tv[GP];
 #pragma unroll
-                            for (int c4 = 0; c4 < GP / 4; ++c4) {
-                                const float4 f = reinterpret_cast<const float4*>(e)[c4];
-                                tv[4 * c4] = f.x; tv[4 * c4 + 1] = f.y; tv[4 * c4 + 2] = f.z; tv[4 * c4 + 3] = f.w;
+                                for (int c4 = 0; c4 < GP / 4; ++c4) {
+                                    const float4 f = reinterpret_cast<const float4*>(e)[c4];
+                                    tv[4 * c4] = f.x; tv[4 * c4 + 1] = f.y; tv[4 * c4 + 2] = f.z; tv[4 * c4 + 3] = f.w;
+                                }
+                                const float x = fmaf(-mu, tv[G], kv);
+#pragma unroll
+                                for (int gg = 0; gg < G; ++gg) a[gg] = fmaf(tv[gg], x, a[gg]);
                             }
-                            const float x = fmaf(-mu, tv[G], kv);
-#pragma unroll
-                            for (int gg = 0; gg < G; ++gg) a[gg] = fmaf(tv[gg], x, a[gg]);
                         }
-                    }
 #pragma unroll
-                    for (int gg = 0; gg < G; ++gg) s[gg] = fmaf(mu, qsum[gg], a[gg]);
+                        for (int gg = 0; gg < G; ++gg) s[gg] = fmaf(mu, qsum[gg], a[gg]);
+                    } else {
+                        // sampled recovery: every channel contributes, kept ones their stored value, pruned
+                        // ones a draw divided by a[j]
+                        const float mean = *reinterpret_cast<const float*>(page + L.stats_off + p * 4);
+                        const float dev = *reinterpret_cast<const float*>(page + L.stats_off + (kPageTokens + p) * 4);
+                        const unsigned long long unit_t =
+                            (static_cast<unsigned long long>(b * A.Hkv + h) << 40) ^
+                            (static_cast<unsigned long long>(i * kStepTokens + lane) << 8);
+#pragma unroll 1
+                        for (int wi = 0; wi < 4; ++wi) {
+                            const unsigned w = words[wi];
+#pragma unroll 4
+                            for (int bp = 0; bp < 32; ++bp) {
+                                const int j = wi * 32 + bp;
+                                const float* e = qtab + j * GP;
+                                float tv[GP];
+#pragma unroll
+                                for (int c4 = 0; c4 < GP / 4; ++c4) {
+                                    const float4 f = reinterpret_cast<const float4*>(e)[c4];
+                                    tv[4 * c4] = f.x; tv[4 * c4 + 1] = f.y; tv[4 * c4 + 2] = f.z; tv[4 * c4 + 3] = f.w;
+                                }
+                                float x;
+                                if ((w >> bp) & 1u) {
+                                    x = kBf16 ? bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(vp))
+                                              : *reinterpret_cast<const float*>(vp);
+                                    vp += kRowBytes;
+                                } else {
+                                    x = sample_saliency<R>(A.seed, unit_t, j, mean, dev) * tv[G];
+                                }
+#pragma unroll
+                                for (int gg = 0; gg < G; ++gg) a[gg] = fmaf(tv[gg], x, a[gg]);
+                            }
+                        }
+#pragma unroll
+                        for (int gg = 0; gg < G; ++gg) s[gg] = a[gg];
+                    }
                 } else {
 #pragma unroll
                     for (int gg = 0; gg < G; ++gg) s[gg] = -INFINITY;
@@ -172,7 +247,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                 for (int t = 0; t < n_valid; ++t) {
                     const unsigned char* pg = sbase + (t >> 4) * L.page_bytes;
                     float vv[4];
-                    if (L.keep_v < kHeadDim) {             // pruned values: this lane's nibble of the value mask
+                    if (!kBf16 && L.keep_v < kHeadDim) {   // pruned values (fp32 pages): this lane's nibble of the value mask
                         const int p = t & 15, wi = lane >> 3, sh = 4 * (lane & 7);
                         const uint4 vm = *reinterpret_cast<const uint4*>(pg + L.vmask_off + p * 16);
                         const unsigned word = wi == 0 ? vm.x : (wi == 1 ? vm.y : (wi == 2 ? vm.z : vm.w));
@@ -186,6 +261,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_f32_kernel(const Dec
                             vv[c] = on ? vb[kPageTokens * slot] : 0.f;
                             slot += on ? 1 : 0;
                         }
+                    } else if (kBf16) {                    // 16-byte chunks of a bf16 value row are stored swizzled
+                        const uint2 r = *reinterpret_cast<const uint2*>(
+                            pg + L.v_off + v_chunk_offset(2, t & 15, lane >> 1) + (lane & 1) * 8);
+                        vv[0] = __uint_as_float(r.x << 16); vv[1] = __uint_as_float(r.x & 0xffff0000u);
+                        vv[2] = __uint_as_float(r.y << 16); vv[3] = __uint_as_float(r.y & 0xffff0000u);
                     } else {
                         const float4 r = *reinterpret_cast<const float4*>(pg + L.v_off + (t & 15) * (kHeadDim * 4) + lane * 16);
                         vv[0] = r.x; vv[1] = r.y; vv[2] = r.z; vv[3] = r.w;
@@ -257,8 +337,8 @@ size_t decode_workspace_bytes(const spark_params& p)
     return align_up(bytes, 256);
 }
 
-template <int G>
-static spark_status launch_f32(const DecodeArgs& A0, int dev, const DeviceInfo& info, cudaStream_t stream)
+template <int G, typename E, int R>
+static spark_status launch_scalar(const DecodeArgs& A0, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
     static unsigned char smem_raised[kMaxDevices] = {};
     const int n_sms = info.n_sms, smem_optin = info.smem_optin;
@@ -273,25 +353,42 @@ static spark_status launch_f32(const DecodeArgs& A0, int dev, const DeviceInfo& 
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
     const size_t smem = A.ring_off + static_cast<size_t>(ns) * A.slot_stride;
-    if (!allow_max_smem(decode_f32_kernel<G>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
+    if (!allow_max_smem(decode_scalar_kernel<G, E, R>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
-    return launch_decode_kernel(decode_f32_kernel<G>, grid, kDecodeThreads, smem, stream, A) == cudaSuccess
+    return launch_decode_kernel(decode_scalar_kernel<G, E, R>, grid, kDecodeThreads, smem, stream, A) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+template <typename E, int R>
+static spark_status launch_scalar_g(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream)
+{
+    switch (G) {
+        case 1: return launch_scalar<1, E, R>(A, dev, info, stream);
+        case 2: return launch_scalar<2, E, R>(A, dev, info, stream);
+        case 3: return launch_scalar<3, E, R>(A, dev, info, stream);
+        case 4: return launch_scalar<4, E, R>(A, dev, info, stream);
+        case 5: return launch_scalar<5, E, R>(A, dev, info, stream);
+        case 6: return launch_scalar<6, E, R>(A, dev, info, stream);
+        case 7: return launch_scalar<7, E, R>(A, dev, info, stream);
+        case 8: return launch_scalar<8, E, R>(A, dev, info, stream);
+        default: return SPARK_ERR_UNSUPPORTED;
+    }
 }
 
 spark_status launch_decode_f32(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
-    switch (G) {
-        case 1: return launch_f32<1>(A, dev, info, stream);
-        case 2: return launch_f32<2>(A, dev, info, stream);
-        case 3: return launch_f32<3>(A, dev, info, stream);
-        case 4: return launch_f32<4>(A, dev, info, stream);
-        case 5: return launch_f32<5>(A, dev, info, stream);
-        case 6: return launch_f32<6>(A, dev, info, stream);
-        case 7: return launch_f32<7>(A, dev, info, stream);
-        case 8: return launch_f32<8>(A, dev, info, stream);
-        default: return SPARK_ERR_UNSUPPORTED;
+    switch (A.L.recovery) {
+        case SPARK_RECOVER_GAUSSIAN: return launch_scalar_g<float, 1>(G, A, dev, info, stream);
+        case SPARK_RECOVER_EXPONENTIAL: return launch_scalar_g<float, 2>(G, A, dev, info, stream);
+        default: return launch_scalar_g<float, 0>(G, A, dev, info, stream);
     }
+}
+
+// bf16 storage with a sampled recovery distribution (the degenerate rule runs on the tensor-core kernel)
+spark_status launch_decode_bf16_sampled(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream)
+{
+    return A.L.recovery == SPARK_RECOVER_GAUSSIAN ? launch_scalar_g<__nv_bfloat16, 1>(G, A, dev, info, stream)
+                                                  : launch_scalar_g<__nv_bfloat16, 2>(G, A, dev, info, stream);
 }
 
 spark_status launch_decode(const spark_params& p, const void* q, const void* pages,
@@ -309,7 +406,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.q = q; A.pages = static_cast<const unsigned char*>(pages); A.block_table = block_table;
     A.max_blocks = max_blocks; A.lens = packed_lens; A.qnorm = qnorm; A.out = out; A.lse = lse;
     A.B = p.batch; A.Hq = p.n_q_heads; A.Hkv = p.n_kv_heads; A.n_pool_pages = p.n_pool_pages;
-    A.L = make_layout(p.dtype, p.keep, p.keep_v);
+    A.L = make_layout(p);
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf(static_cast<float>(p.head_dim));
     A.scale_log2e = scale * 1.4426950408889634f;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -318,8 +415,10 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.partials = reinterpret_cast<float*>(ws + kWorkspaceHeader + align_up(units * sizeof(int), 256));
     A.nslots = 0; A.slot_stride = 0; A.pps = 1; A.prefix_off = 0; A.ring_off = 0;
     A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
-    const spark_status st = (p.dtype == SPARK_BF16) ? launch_decode_bf16(G, A, dev, info, stream)
-                                                    : launch_decode_f32(G, A, dev, info, stream);
+    A.seed = p.seed;
+    const spark_status st = (p.dtype != SPARK_BF16) ? launch_decode_f32(G, A, dev, info, stream)
+                            : (p.recovery != SPARK_RECOVER_DEGENERATE) ? launch_decode_bf16_sampled(G, A, dev, info, stream)
+                                                                       : launch_decode_bf16(G, A, dev, info, stream);
     if (st == SPARK_OK) ++*launches;
     return st;
 }

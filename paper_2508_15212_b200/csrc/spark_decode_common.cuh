@@ -43,6 +43,7 @@ struct DecodeArgs {
     int prefix_off;                          // shared-memory offset of the steps-per-sequence prefix ((B + 1) ints)
     int ring_off;                            // shared-memory offset of the ring (behind the prefix)
     int overlap;                             // launched as a programmatic dependent of the preceding kernel
+    unsigned seed;                           // sampled recovery: seed of the per-entry draws
 };
 
 // control block at the start of dynamic shared memory
@@ -667,5 +668,6 @@ template <typename Kernel> inline bool allow_max_smem(Kernel kernel, int dev, in
 // per-dtype launchers (spark_decode.cu: fp32 storage, spark_decode_mma.cu: bf16 storage)
 spark_status launch_decode_f32(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream);
 spark_status launch_decode_bf16(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream);
+spark_status launch_decode_bf16_sampled(int G, const DecodeArgs& A, int dev, const DeviceInfo& info, cudaStream_t stream);
 
 }  // namespace spark
