@@ -125,23 +125,39 @@ def workload_desc(cfg, keep, copies=None, keep_v=0):
 # ----------------------------------------------------------------------------------------------------
 # the oracle on the host cores
 # ----------------------------------------------------------------------------------------------------
-def oracle_prepare(q_win, k, v, lens, keep, keep_v=0):
-    """Untimed preparation of an oracle decode: window mean, key pruning, value masks."""
+def oracle_prepare(q_win, k, v, lens, keep, keep_v=0, variant=None):
+    """Untimed preparation of an oracle decode: window mean, key pruning (fixed T or a ratio-free variant),
+    value masks.  `variant` = dict(top_p | group_prune, recovery, seed) or None."""
     import oracle
+    variant = variant or {}
     _, a = oracle.window_mean(q_win, k.shape[1])
-    c = oracle.compress(k, lens, keep, a)
+    if variant.get("top_p") is not None:
+        c = oracle.select_variant(k, lens, a, top_p=variant["top_p"], cap=keep, want_stats=True)
+    elif variant.get("group_prune") is not None:
+        c = oracle.select_variant(k, lens, a, group_prune=variant["group_prune"], want_stats=True)
+    else:
+        c = oracle.compress(k, lens, keep, a, want_stats=bool(variant.get("recovery")))
+    c["recovery"], c["seed"] = int(variant.get("recovery") or 0), int(variant.get("seed") or 0)
     vm = oracle.prune_values(v, lens, keep_v) if 0 < keep_v < 128 else None
     return a, c, vm
+
+
+def oracle_decode(q, k, v, lens, a, c, vm):
+    import oracle
+    if c.get("recovery"):
+        return oracle.decode_attn_sampled(q, k, v, lens, c["mask"], c["mu_all"], c["sigma_all"], a,
+                                          mode=c["recovery"], seed=c["seed"])[0]
+    return oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, vmask=vm)[0]
 
 
 def oracle_decode_time(q, k, v, lens, a, c, vm, reps=3):
     """Median time of the oracle's decode step on the host cores -> (seconds, threads, output)."""
     import oracle
-    oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, vmask=vm)                   # warm
+    oracle_decode(q, k, v, lens, a, c, vm)                                               # warm
     ts, out = [], None
     for _ in range(reps):
         t0 = time.perf_counter()
-        out, _ = oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, vmask=vm)
+        out = oracle_decode(q, k, v, lens, a, c, vm)
         ts.append(time.perf_counter() - t0)
     return statistics.median(ts), oracle.threads(), out
 
@@ -195,19 +211,21 @@ class Work:
         self.oracle_inputs = None          # callable -> (q, k, v, lens, q_win) host tensors of set 0, or None
         self.oracle_sample = None
         self.cfg, self.keep, self.keep_v = None, 0, 0
+        self.variant = None                # dict(top_p | group_prune, recovery, seed) of a ratio-free / sampled run
 
     @property
     def launches_per_step(self):
         return len(self.step_sets[0])
 
 
-def build_work(index, cfg, keep, keep_v, rank, torch, B):
+def build_work(index, cfg, keep, keep_v, rank, torch, B, variant=None):
     from paper_2508_15212_b200 import dist_utils
     from paper_2508_15212_b200.cache import SparkCache
     from workloads import inputs
     from workloads.batches import build_evicted_batch, permuted_block_table
     w = Work()
-    w.cfg, w.keep, w.keep_v = cfg, keep, keep_v
+    w.cfg, w.keep, w.keep_v, w.variant = cfg, keep, keep_v, variant
+    vkw = {} if not variant else {k_: v_ for k_, v_ in variant.items() if v_ is not None}
     l2 = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size
     D = cfg["head_dim"]
     esize = 2 if cfg["dtype"] == "bf16" else 4
@@ -262,7 +280,7 @@ def build_work(index, cfg, keep, keep_v, rank, torch, B):
         Bn, Hq, Hkv, W, _, S = wl.shape
         lens = wl.seq_lens.tolist()
         mk = lambda: SparkCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, window=W, keep=keep, dtype=wl.dtype,
-                                max_tokens=S, keep_v=keep_v)
+                                max_tokens=S, keep_v=keep_v, **vkw)
         first = mk()
         w.alg_bytes = first.algorithmic_bytes_per_token * Hkv * sum(lens)
         w.copies = max(1, min(64, -(-4 * l2 // max(w.alg_bytes, 1))))
@@ -366,7 +384,7 @@ def oracle_check(work):
     if work.oracle_inputs is None:
         return None, None, None
     q, k, v, lens, q_win = work.oracle_inputs()
-    a, c, vm = oracle_prepare(q_win, k, v, lens, work.keep, work.keep_v)
+    a, c, vm = oracle_prepare(q_win, k, v, lens, work.keep, work.keep_v, work.variant)
     t_or, cores, o_ref = oracle_decode_time(q, k, v, lens, a, c, vm)
     cache, qd, _ = work.step_sets[0][0]
     for cch in work.caches:
@@ -389,7 +407,7 @@ def oracle_single_thread(prepared, cores):
     omp.omp_set_num_threads(1)
     try:
         t0 = time.perf_counter()
-        oracle.decode_attn(q, k, v, lens, c["mask"], c["mu"], a, vmask=vm)
+        oracle_decode(q, k, v, lens, a, c, vm)
         dt = time.perf_counter() - t0
     finally:
         omp.omp_set_num_threads(int(cores))
@@ -408,6 +426,12 @@ def main():
     ap.add_argument("--ratio", type=float, default=None, help="pruning ratio (configuration 5 sweeps 0.3/0.5/0.7/0.8)")
     ap.add_argument("--ratio-v", type=float, default=None,
                     help="also prune value channels with this ratio (default: values stay dense)")
+    ap.add_argument("--top-p", type=float, default=None, help="SparK-p: keep the channels that reach this share of a "
+                    "token's saliency (the page holds up to --keep, default 128, channels per token)")
+    ap.add_argument("--groups", type=str, default=None, help="SparK-g: comma-separated pruning ratios of the rank "
+                    "groups, most salient first (e.g. 0.25,0.5,0.75,1.0)")
+    ap.add_argument("--recovery", default="degenerate", choices=["degenerate", "gaussian", "exponential"])
+    ap.add_argument("--seed", type=int, default=1, help="seed of the sampled-recovery draws")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="time only the workload named by --config")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
@@ -458,12 +482,23 @@ def main():
     cfg, keep = resolve(args.config, args.ratio, args.batch)
     keep = args.keep or keep
     keep_v = B.spark_keep_count(cfg["head_dim"], args.ratio_v) if args.ratio_v is not None else 0
+    variant = None
+    recovery = {"degenerate": 0, "gaussian": 1, "exponential": 2}[args.recovery]
+    if args.top_p is not None or args.groups or recovery:
+        groups = [float(x) for x in args.groups.split(",")] if args.groups else None
+        variant = dict(top_p=args.top_p, group_prune=groups, recovery=recovery, seed=args.seed if recovery else 0)
+        if groups:
+            keep = B.spark_group_keep(cfg["head_dim"], groups)
+        elif args.top_p is not None:
+            keep = args.keep or cfg["head_dim"]
+        if "token_budget" in cfg or "n_layers" in cfg:
+            raise SystemExit("the variant flags are wired for the single-layer configurations (0, 1, 2)")
     stream = torch.cuda.Stream()
     sampler = ClockSampler(local)
     peak, peak_kind = measured_peak()
 
     # ---- the headline workload ----
-    work = build_work(args.config, cfg, keep, keep_v, rank, torch, B)
+    work = build_work(args.config, cfg, keep, keep_v, rank, torch, B, variant)
     first = work.caches[0]
     t_plain = time_work(work, args.steps, args.warmup, 0, dist, torch, stream, sampler)
     t_pdl = time_work(work, args.steps, args.warmup, B.SPARK_FLAG_OVERLAP_PREVIOUS, dist, torch, stream, sampler)
@@ -511,7 +546,8 @@ def main():
 
     # ---- the other workloads of the target range (N = 1, default configuration only) ----
     sweep = []
-    if world == 1 and args.config == 1 and not args.no_sweep and not keep_v and not args.batch and not args.keep:
+    if world == 1 and args.config == 1 and not args.no_sweep and not keep_v and not args.batch and not args.keep \
+            and variant is None:
         for idx in (2, 3):
             torch.cuda.empty_cache()
             cfg_s, keep_s = resolve(idx)
@@ -542,7 +578,8 @@ def main():
             "warmup": max(args.warmup, 3), "ms_per_step": us_step / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": cfg["dtype"], "data": "synthetic",
             "config": dict(workload_desc(cfg, keep, work.copies, keep_v),
-                           launch="ordinary launches, K steps replayed from CUDA graphs"),
+                           launch="ordinary launches, K steps replayed from CUDA graphs",
+                           **({"variant": {k_: v_ for k_, v_ in variant.items() if v_}} if variant else {})),
             "replays": {"n": t_plain["replays"], "steps_per_replay": t_plain["steps_per_replay"],
                         "median_us_per_step": t_plain["median_us"], "min_us_per_step": t_plain["min_us"]},
             "value_pdl": t_pdl["us_step"],
@@ -561,7 +598,8 @@ def main():
             "launches_per_step": lps,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(name) if not keep_v else None,
-                         "kernel": "spark::decode_bf16_kernel" if cfg["dtype"] == "bf16" else "spark::decode_f32_kernel",
+                         "kernel": ("spark::decode_bf16_kernel" if cfg["dtype"] == "bf16" and not recovery
+                                    else "spark::decode_scalar_kernel"),
                          "algorithmic_bytes_per_launch": work.alg_bytes / lps,
                          "avg_launch_us": us_step / lps},
             "cpu_baseline": cpu_baseline,
