@@ -212,6 +212,32 @@ spark_status spark_append(const spark_params *p, const void *k_new, const void *
                           void *workspace, size_t workspace_bytes, spark_stream_t stream);
 
 /*
+ * spark_append_block -- the same for n_new tokens per sequence at once: k_new, v_new are [B][Hkv][n_new][D]
+ * and every sequence grows by n_new tokens (by as many as fit; SPARK_ERR_DEVICE_BOUNDS is recorded when some do
+ * not).  This is how keys that a caller has kept DENSE for a while -- the paper's K <- Cat[K, k] of Sec.
+ * "Preliminaries" taken literally -- enter the pruned cache block by block.  0 <= n_new <= 65535.
+ */
+spark_status spark_append_block(const spark_params *p, const void *k_new, const void *v_new, int32_t n_new,
+                                void *pages, const int32_t *block_table, int32_t max_blocks,
+                                const float *qnorm, int32_t *packed_lens,
+                                void *workspace, size_t workspace_bytes, spark_stream_t stream);
+
+/*
+ * spark_merge_attn -- attention over the union of two disjoint token sets from the two partial results
+ * (Sec. "Preliminaries": softmax attention; the log-sum-exp identity that also merges the token splits inside
+ * spark_decode_attn).  With w_x = exp(lse_x - lse), lse = log(exp(lse_a) + exp(lse_b)):
+ *     out = w_a * out_a + w_b * out_b
+ * A side with lse = -inf (no tokens) contributes nothing; both empty gives out = 0, lse = -inf.  Typical use:
+ * a sequence held as a pruned prefix (one cache) plus a dense tail of recently appended tokens (a second cache
+ * with keep = head_dim): decode both with their lse and merge.
+ *   out_a, out_b, out  [batch][n_q_heads][head_dim] fp32, 16-byte aligned (out may alias an input)
+ *   lse_a, lse_b       [batch][n_q_heads] fp32;  lse  OUT optional
+ */
+spark_status spark_merge_attn(int32_t batch, int32_t n_q_heads, int32_t head_dim,
+                              const float *out_a, const float *lse_a, const float *out_b, const float *lse_b,
+                              float *out, float *lse, spark_stream_t stream);
+
+/*
  * spark_decode_attn -- one decode step over the packed cache (Sec. "Channel Recovery"
  * with the degenerate distribution, then the attention of Sec. "Preliminaries").
  *

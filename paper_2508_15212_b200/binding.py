@@ -22,7 +22,7 @@ SPARK_F32, SPARK_BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
 EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
-           "spark_compress", "spark_append", "spark_decode_attn", "spark_decode_attn_host", "spark_decode_attn_noalloc", "spark_unpack_pages",
+           "spark_compress", "spark_append", "spark_append_block", "spark_merge_attn", "spark_decode_attn", "spark_decode_attn_host", "spark_decode_attn_noalloc", "spark_unpack_pages",
            "spark_unpack_value_masks", "spark_unpack_stats", "spark_group_keep", "spark_read_status"]
 
 
@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.spark_compress.argtypes = [P, vp, vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.spark_append.restype = i32
         L.spark_append.argtypes = [P, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.spark_append_block.restype = i32
+        L.spark_append_block.argtypes = [P, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.spark_merge_attn.restype = i32
+        L.spark_merge_attn.argtypes = [i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.spark_decode_attn.restype = i32
         L.spark_decode_attn.argtypes = [P, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.spark_decode_attn_host.restype = i32
@@ -191,6 +195,25 @@ def spark_append(p: spark_params, k_new, v_new, pages, block_table, qnorm, packe
                               _blocks(block_table, max_blocks), _ptr(qnorm), _ptr(packed_lens), _ptr(workspace),
                               workspace.numel() * workspace.element_size(), _stream()),
            "spark_append")
+
+
+def spark_append_block(p: spark_params, k_new, v_new, pages, block_table, qnorm, packed_lens, workspace,
+                       max_blocks=None) -> None:
+    """k_new, v_new: [B, Hkv, n_new, D] contiguous; every sequence grows by n_new tokens."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape and k_new.dim() == 4
+    _check(lib().spark_append_block(ctypes.byref(p), _ptr(k_new), _ptr(v_new), int(k_new.shape[2]), _ptr(pages),
+                                    _ptr(block_table), _blocks(block_table, max_blocks), _ptr(qnorm),
+                                    _ptr(packed_lens), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream()),
+           "spark_append_block")
+
+
+def spark_merge_attn(out_a, lse_a, out_b, lse_b, out, lse=None) -> None:
+    """Merge two partial attention results ([B, Hq, 128] fp32 with their [B, Hq] log-sum-exp)."""
+    Bn, Hq, D = out_a.shape
+    _check(lib().spark_merge_attn(Bn, Hq, D, _ptr(out_a), _ptr(lse_a), _ptr(out_b), _ptr(lse_b), _ptr(out), _ptr(lse),
+                                  _stream()),
+           "spark_merge_attn")
 
 
 def spark_decode_attn(p: spark_params, q, pages, block_table, packed_lens, qnorm, out, lse, workspace,

@@ -101,6 +101,11 @@ class SparkCache:
         B.spark_append(self.params, k_new, v_new, self.pages, self.block_table, self.qnorm, self.packed_lens,
                        self.ws_compress, max_blocks=self.table_blocks)
 
+    def append_block(self, k_new, v_new) -> None:
+        """n new tokens per sequence ([B, Hkv, n, D]), each pruned with the prefill statistics."""
+        B.spark_append_block(self.params, k_new, v_new, self.pages, self.block_table, self.qnorm, self.packed_lens,
+                             self.ws_compress, max_blocks=self.table_blocks)
+
     def decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
         p = self.params
         if out is None:
@@ -155,3 +160,61 @@ class SparkCache:
     @property
     def algorithmic_bytes_per_token(self) -> int:
         return B.spark_algorithmic_bytes_per_token(self.params)
+
+
+class DenseTailCache:
+    """A sequence held as a pruned prefix plus a DENSE tail of recently appended tokens.
+
+    The paper appends the keys of generated tokens as they are (K <- Cat[K, k], Sec. "Preliminaries") and prunes
+    "during prefill"; this object is that reading.  Appended tokens go, unpruned, into a small second cache whose
+    pages keep all 128 channels; every `tail_block` appended tokens the dense copies that this object also keeps
+    are handed to the prefix in one spark_append_block call (pruned with the prefill statistics) and the tail
+    starts over.  `tail_block=None` never hands them over: the literal "dense appended keys".  A decode step is
+    the prefix step, the tail step and their log-sum-exp merge (spark_merge_attn); all arithmetic is in the
+    library.
+    """
+
+    def __init__(self, *, batch: int, n_q_heads: int, n_kv_heads: int, window: int, keep: int, dtype: str,
+                 max_tokens: int, tail_block: Optional[int] = 64, max_tail: int = 1024, device="cuda", **prefix_kw):
+        self.block = int(tail_block) if tail_block else None
+        cap = self.block if self.block else int(max_tail)
+        self.prefix = SparkCache(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window, keep=keep,
+                                 dtype=dtype, max_tokens=max_tokens, device=device, **prefix_kw)
+        self.tail = SparkCache(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, window=window, keep=128,
+                               dtype=dtype, max_tokens=cap, device=device)
+        tdt = _TDT[dtype]
+        self.k_tail = torch.zeros(batch, n_kv_heads, cap, 128, dtype=tdt, device=device)
+        self.v_tail = torch.zeros(batch, n_kv_heads, cap, 128, dtype=tdt, device=device)
+        self.n_tail = 0
+        p = self.prefix.params
+        self._o = [torch.empty(p.batch, p.n_q_heads, 128, dtype=torch.float32, device=device) for _ in range(2)]
+        self._l = [torch.empty(p.batch, p.n_q_heads, dtype=torch.float32, device=device) for _ in range(2)]
+
+    def compress(self, q_win, k, v, seq_lens) -> None:
+        self.prefix.compress(q_win, k, v, seq_lens)
+        self.tail.qnorm.copy_(self.prefix.qnorm)           # the tail is dense: qnorm only has to be a valid divisor
+        self.tail.packed_lens.zero_()
+        self.n_tail = 0
+
+    def append(self, k_new, v_new) -> None:
+        """One new token per sequence ([B, Hkv, D]); it stays dense until its block is handed to the prefix."""
+        self.tail.append(k_new, v_new)
+        self.k_tail[:, :, self.n_tail].copy_(k_new)
+        self.v_tail[:, :, self.n_tail].copy_(v_new)
+        self.n_tail += 1
+        if self.block and self.n_tail == self.block:
+            self.prefix.append_block(self.k_tail, self.v_tail)
+            self.tail.packed_lens.zero_()
+            self.n_tail = 0
+
+    def decode(self, q, out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None):
+        if out is None:
+            out = torch.empty_like(self._o[0])
+        self.prefix.decode(q, out=self._o[0], lse=self._l[0])
+        self.tail.decode(q, out=self._o[1], lse=self._l[1])
+        B.spark_merge_attn(self._o[0], self._l[0], self._o[1], self._l[1], out, lse)
+        return out
+
+    def status(self) -> int:
+        s = self.prefix.status()
+        return s if s else self.tail.status()

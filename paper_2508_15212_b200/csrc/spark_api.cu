@@ -173,6 +173,36 @@ spark_status spark_append(const spark_params* p, const void* k_new, const void* 
     return st;
 }
 
+spark_status spark_append_block(const spark_params* p, const void* k_new, const void* v_new, int32_t n_new,
+                                void* pages, const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                                int32_t* packed_lens, void* workspace, size_t workspace_bytes, spark_stream_t stream)
+{
+    spark_status st = check_params(p);
+    if (st != SPARK_OK) return st;
+    if (!k_new || !v_new || !pages || !qnorm || !packed_lens || !workspace) return SPARK_ERR_NULL;
+    if (max_blocks < 1 || max_blocks > kMaxBlocksArg || n_new < 0 || n_new > 65535) return SPARK_ERR_BAD_SHAPE;
+    if (contiguous_pool_too_small(p, block_table, max_blocks)) return SPARK_ERR_BAD_SHAPE;
+    if (misaligned(pages, 16) || misaligned(k_new, 16) || misaligned(v_new, 16) || misaligned(qnorm, 16))
+        return SPARK_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < kWorkspaceHeader) return SPARK_ERR_WORKSPACE;
+    int launches = 0;
+    st = launch_append_block(*p, k_new, v_new, n_new, pages, block_table, max_blocks, qnorm, packed_lens, workspace,
+                             static_cast<cudaStream_t>(stream), &launches);
+    if (st == SPARK_OK) g_last_launches = launches;
+    return st;
+}
+
+spark_status spark_merge_attn(int32_t batch, int32_t n_q_heads, int32_t head_dim, const float* out_a,
+                              const float* lse_a, const float* out_b, const float* lse_b, float* out, float* lse,
+                              spark_stream_t stream)
+{
+    if (!out_a || !lse_a || !out_b || !lse_b || !out) return SPARK_ERR_NULL;
+    if (head_dim != kHeadDim) return SPARK_ERR_UNSUPPORTED;
+    if (batch < 0 || n_q_heads < 0 || static_cast<int64_t>(batch) * n_q_heads > INT32_MAX) return SPARK_ERR_BAD_SHAPE;
+    if (misaligned(out_a, 16) || misaligned(out_b, 16) || misaligned(out, 16)) return SPARK_ERR_BAD_SHAPE;
+    return launch_merge_attn(batch * n_q_heads, out_a, lse_a, out_b, lse_b, out, lse, static_cast<cudaStream_t>(stream));
+}
+
 spark_status spark_decode_attn(const spark_params* p, const void* q, const void* pages,
                                const int32_t* block_table, int32_t max_blocks,
                                const int32_t* packed_lens, const float* qnorm, float* out, float* lse,

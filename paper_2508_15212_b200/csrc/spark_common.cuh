@@ -127,6 +127,12 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
                            const int32_t* block_table, int32_t max_blocks, const float* qnorm,
                            int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches);
 
+spark_status launch_append_block(const spark_params& p, const void* k_new, const void* v_new, int32_t n_new,
+                                 void* pages, const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                                 int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches);
+spark_status launch_merge_attn(int rows, const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
+                               float* out, float* lse, cudaStream_t stream);
+
 size_t decode_workspace_bytes(const spark_params& p);
 size_t evict_workspace_bytes(const spark_params& p, int64_t max_seq_tokens);
 spark_status launch_evict(const spark_params& p, const void* q_win, const void* k, int64_t sb, int64_t sh,

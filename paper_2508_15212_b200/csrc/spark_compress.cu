@@ -451,6 +451,72 @@ __global__ void append_advance_kernel(AppendArgs A)
     if (t >= 0 && t / kPageTokens < A.max_blocks) A.packed_lens[b] = t + 1;
 }
 
+// Block append: n_new tokens per sequence at once (the keys a caller has kept dense for a while and now hands
+// over for pruning).  Three launches: fresh pages are zeroed, every (sequence, head, new token) gets a warp that
+// prunes it exactly like append_token_kernel, packed_lens advances by the tokens that found room.
+struct AppendBlockArgs {
+    AppendArgs a;
+    int n_new;
+};
+
+__global__ void __launch_bounds__(32) append_block_clear_kernel(AppendBlockArgs B_)
+{
+    const AppendArgs& A = B_.a;
+    const int h = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+    const int t0 = A.packed_lens[b];
+    if (t0 < 0) return;
+    const int blk = (t0 + kPageTokens - 1) / kPageTokens + static_cast<int>(blockIdx.z);   // pages that start at or after t0
+    if (static_cast<int64_t>(blk) * kPageTokens >= static_cast<int64_t>(t0) + B_.n_new || blk >= A.max_blocks) return;
+    const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+    const int64_t page_id = A.block_table ? A.block_table[entry] : entry;
+    if (page_id < 0 || page_id >= A.n_pool_pages) {
+        if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    uint4* page = reinterpret_cast<uint4*>(A.pages + page_id * A.L.page_bytes);
+    for (int i = lane; i < A.L.page_bytes / 16; i += 32) page[i] = make_uint4(0, 0, 0, 0);
+}
+
+template <typename E>
+__global__ void __launch_bounds__(32) append_block_token_kernel(AppendBlockArgs B_)
+{
+    constexpr bool kBf16 = (sizeof(E) == 2);
+    const AppendArgs& A = B_.a;
+    const int h = blockIdx.x, b = blockIdx.y, tok = blockIdx.z, lane = threadIdx.x;
+    const PageLayout L = A.L;
+    const int t0 = A.packed_lens[b];
+    const int64_t t = static_cast<int64_t>(t0) + tok;
+    const int64_t blk = t / kPageTokens;
+    const int p = static_cast<int>(t - blk * kPageTokens);
+    if (t0 < 0 || blk >= A.max_blocks) {                      // no room: recorded, nothing written
+        if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+    const int64_t page_id = A.block_table ? A.block_table[entry] : entry;
+    if (page_id < 0 || page_id >= A.n_pool_pages) {
+        if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    unsigned char* page = A.pages + page_id * L.page_bytes;
+    const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
+    const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+    const int64_t row = ((static_cast<int64_t>(b) * A.Hkv + h) * B_.n_new + tok) * kHeadDim + lane * 4;
+    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+}
+
+__global__ void append_block_advance_kernel(AppendBlockArgs B_)
+{
+    const AppendArgs& A = B_.a;
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= A.B) return;
+    const int t = A.packed_lens[b];
+    if (t < 0) return;
+    const int64_t room = static_cast<int64_t>(A.max_blocks) * kPageTokens;
+    const int64_t want = static_cast<int64_t>(t) + B_.n_new;
+    A.packed_lens[b] = static_cast<int>(want < room ? want : (t > room ? t : room));
+}
+
 // selection arguments of a parameter block (the rank mask of SparK-g is laid out on the host)
 static SelectArgs make_select(const spark_params& p)
 {
@@ -485,6 +551,65 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     else append_token_kernel<float><<<grid, 32, 0, stream>>>(A);
     append_advance_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(A);
     *launches += 2;
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+spark_status launch_append_block(const spark_params& p, const void* k_new, const void* v_new, int32_t n_new,
+                                 void* pages, const int32_t* block_table, int32_t max_blocks, const float* qnorm,
+                                 int32_t* packed_lens, void* workspace, cudaStream_t stream, int* launches)
+{
+    if (n_new == 0) return SPARK_OK;
+    AppendBlockArgs Bk;
+    AppendArgs& A = Bk.a;
+    A.k_new = k_new; A.v_new = v_new; A.pages = static_cast<unsigned char*>(pages); A.block_table = block_table;
+    A.max_blocks = max_blocks; A.B = p.batch; A.Hkv = p.n_kv_heads; A.keep = p.keep; A.n_pool_pages = p.n_pool_pages;
+    A.L = make_layout(p); A.qnorm = qnorm; A.packed_lens = packed_lens;
+    A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
+    A.sel = make_select(p);
+    A.status = static_cast<int*>(workspace);
+    Bk.n_new = n_new;
+    const int fresh = (n_new + kPageTokens - 1) / kPageTokens + 1;       // pages that can start inside the new tokens
+    append_block_clear_kernel<<<dim3(p.n_kv_heads, p.batch, fresh), 32, 0, stream>>>(Bk);
+    const dim3 grid(p.n_kv_heads, p.batch, n_new);
+    if (p.dtype == SPARK_BF16) append_block_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(Bk);
+    else append_block_token_kernel<float><<<grid, 32, 0, stream>>>(Bk);
+    append_block_advance_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(Bk);
+    *launches += 3;
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Two partial attention results over disjoint token sets -> the result over their union (the log-sum-exp
+// merge that split decoding uses, exposed for callers that hold a sequence in more than one cache).
+// One warp per (sequence, query head) row; lane l owns channels 4l .. 4l+3.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) merge_attn_kernel(int rows, const float* __restrict__ out_a, const float* __restrict__ lse_a,
+                                                         const float* __restrict__ out_b, const float* __restrict__ lse_b,
+                                                         float* __restrict__ out, float* __restrict__ lse)
+{
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const float la = lse_a[row], lb = lse_b[row];
+    const float m = fmaxf(la, lb);
+    float wa = 0.f, wb = 0.f, l = -INFINITY;
+    if (m > -INFINITY) {                                       // at least one side saw tokens
+        const float ea = expf(la - m), eb = expf(lb - m);
+        const float inv = 1.0f / (ea + eb);
+        wa = ea * inv; wb = eb * inv;
+        l = m + logf(ea + eb);
+    }
+    const float4 a = reinterpret_cast<const float4*>(out_a + static_cast<int64_t>(row) * kHeadDim)[lane];
+    const float4 b = reinterpret_cast<const float4*>(out_b + static_cast<int64_t>(row) * kHeadDim)[lane];
+    reinterpret_cast<float4*>(out + static_cast<int64_t>(row) * kHeadDim)[lane] =
+        make_float4(fmaf(wa, a.x, wb * b.x), fmaf(wa, a.y, wb * b.y), fmaf(wa, a.z, wb * b.z), fmaf(wa, a.w, wb * b.w));
+    if (lane == 0 && lse) lse[row] = l;
+}
+
+spark_status launch_merge_attn(int rows, const float* out_a, const float* lse_a, const float* out_b, const float* lse_b,
+                               float* out, float* lse, cudaStream_t stream)
+{
+    if (rows == 0) return SPARK_OK;
+    merge_attn_kernel<<<(rows + 3) / 4, 128, 0, stream>>>(rows, out_a, lse_a, out_b, lse_b, out, lse);
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
 

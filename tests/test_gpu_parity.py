@@ -348,6 +348,80 @@ def test_append_tokens_equals_compressing_the_longer_sequence(dtype, keep):
     assert small.packed_lens.cpu().tolist() == [16] and B.spark_read_status(small.ws_compress) == 6
 
 
+def test_block_append_equals_appending_one_token_at_a_time():
+    lens0, n = [37, 530, 16], 45
+    full = make("bf16", 3, 8, 2, [l + n for l in lens0], 8, 38, seed=152)
+    S = max(lens0) + n
+    lens0_t = torch.tensor(lens0, dtype=torch.int32, device="cuda")
+    idx = (lens0_t.long().view(3, 1, 1, 1) + torch.arange(n, device="cuda").view(1, 1, n, 1)).expand(3, 2, n, 128)
+    k_blk, v_blk = full.k.gather(2, idx).contiguous(), full.v.gather(2, idx).contiguous()
+    one, blk = (SparkCache(batch=3, n_q_heads=8, n_kv_heads=2, window=8, keep=38, dtype="bf16", max_tokens=S,
+                           guard=True) for _ in range(2))
+    for c in (one, blk):
+        c.compress(full.q_win, full.k, full.v, lens0_t)
+    for i in range(n):
+        one.append(k_blk[:, :, i].contiguous(), v_blk[:, :, i].contiguous())
+    blk.append_block(k_blk, v_blk)
+    assert one.status() == 0 and blk.status() == 0 and blk.broken_guards() == []
+    assert blk.packed_lens.cpu().tolist() == [l + n for l in lens0]
+    ua, ub = one.unpack(), blk.unpack()
+    for key in ("mask", "mu", "vals", "v"):
+        assert torch.equal(ua[key], ub[key]), key
+    # more tokens than there is room for: the sequence is filled up and the condition recorded
+    small = SparkCache(batch=1, n_q_heads=4, n_kv_heads=1, window=8, keep=38, dtype="bf16", max_tokens=32)
+    w1 = make("bf16", 1, 4, 1, [40], 8, 38, seed=153, gap=False)
+    small.compress(w1.q_win, w1.k[:, :, :20].contiguous(), w1.v[:, :, :20].contiguous(), torch.tensor([20], dtype=torch.int32, device="cuda"))
+    small.append_block(w1.k[:, :, 20:40].contiguous(), w1.v[:, :, 20:40].contiguous())
+    assert small.packed_lens.cpu().tolist() == [32] and B.spark_read_status(small.ws_compress) == 6
+
+
+@pytest.mark.parametrize("dtype,block,n_app", [("bf16", 16, 41), ("bf16", None, 30), ("f32", 8, 19)])
+def test_dense_tail_equals_the_oracle_with_appended_keys_left_dense(dtype, block, n_app):
+    """Pruned prefix + dense tail (the paper's literal K <- Cat[K, k]): the oracle attends over all tokens with
+    the prefill-pruned mask on the prefix (handed-over blocks included) and every channel kept on the tail."""
+    from paper_2508_15212_b200.cache import DenseTailCache
+    keep, lens0 = 38, [50, 200]
+    full = make(dtype, 2, 8, 2, [l + n_app for l in lens0], 8, keep, seed=160, sigma=1.0 if dtype == "bf16" else 0.5)
+    S = max(lens0) + n_app
+    cache = DenseTailCache(batch=2, n_q_heads=8, n_kv_heads=2, window=8, keep=keep, dtype=dtype, max_tokens=S,
+                           tail_block=block, max_tail=64)
+    lens0_t = torch.tensor(lens0, dtype=torch.int32, device="cuda")
+    cache.compress(full.q_win, full.k, full.v, lens0_t)
+    wl_cpu = full.to("cpu")
+    _, a = oracle.window_mean(wl_cpu.q_win, 2)
+    c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a)
+    for i in range(n_app):
+        idx = (lens0_t.long() + i).view(2, 1, 1, 1).expand(2, 2, 1, 128)
+        cache.append(full.k.gather(2, idx).squeeze(2).contiguous(), full.v.gather(2, idx).squeeze(2).contiguous())
+        if i in (0, n_app // 2, n_app - 1):
+            n_dense = (i + 1) if block is None else (i + 1) % block
+            mask, mu, lens_now = c["mask"].copy(), c["mu"].copy(), [l + i + 1 for l in lens0]
+            for b, l in enumerate(lens_now):                 # the last n_dense tokens are still dense
+                mask[b, :, l - n_dense:l] = 0xFFFFFFFF
+                mu[b, :, l - n_dense:l] = 0.0
+            ref, ref_lse = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, lens_now, mask, mu, a)
+            lse = torch.empty(2, 8, dtype=torch.float32, device="cuda")
+            out = cache.decode(full.q, lse=lse)
+            assert cache.status() == 0
+            d = float(np.abs(out.cpu().numpy() - ref).max())
+            assert d <= TOL[dtype], f"after {i + 1} appended tokens: max|delta| {d:.3e}"
+            assert np.allclose(lse.cpu().numpy(), ref_lse, rtol=0, atol=1e-3 if dtype == "bf16" else 2e-5)
+
+
+def test_merge_attn_handles_empty_sides():
+    o = torch.randn(2, 4, 128, device="cuda")
+    zero = torch.zeros_like(o)
+    l = torch.tensor([[0.5, -1.0, 2.0, 0.0]] * 2, device="cuda")
+    ninf = torch.full_like(l, float("-inf"))
+    out, lse = torch.empty_like(o), torch.empty_like(l)
+    B.spark_merge_attn(o, l, zero, ninf, out, lse)
+    assert torch.equal(out, o) and torch.equal(lse, l)
+    B.spark_merge_attn(zero, ninf, zero, ninf, out, lse)
+    assert bool((out == 0).all()) and bool(torch.isneginf(lse).all())
+    B.spark_merge_attn(o, l, o, l, out, lse)                    # equal halves: same output, lse + ln 2
+    assert torch.allclose(out, o, atol=1e-6) and torch.allclose(lse, l + 0.6931472, atol=1e-6)
+
+
 # ---- value-channel pruning (App. "Pruning Value Cache Channels") ------------------------------------
 @pytest.mark.parametrize("keep,keep_v", [(64, 64), (64, 89), (25, 25), (38, 1), (128, 64), (64, 127)])
 def test_value_pruning_bf16_ragged(keep, keep_v):
