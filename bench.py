@@ -39,7 +39,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the ncu captures summarised in
 # profiles/decode_bf16_*.md (bytes)
-NCU_TRAFFIC_BYTES = {"llama8b_32k": 109.3e6, "llama8b_4x128k": 1391.7e6}
+NCU_TRAFFIC_BYTES = {"llama8b_32k": 109.6e6, "llama8b_4x128k": 1380.6e6}        # 4 x (342.0 + 3.16) MB from one 128K sequence
 MIN_REPLAYS = 50
 
 
