@@ -132,6 +132,12 @@ int32_t spark_group_keep(int32_t head_dim, int32_t n_groups, const float *group_
  * Host only.  0 on unsupported parameters. */
 size_t spark_page_bytes(const spark_params *p);
 
+/* Bytes of the whole page pool: n_pool_pages * spark_page_bytes(p), plus -- under SPARK_SELECT_TOP_P -- an
+ * int32 per pool page behind the pages (256-byte aligned) in which the library keeps how many slot rows of
+ * the page are in use; the decode step then copies only that much of each page.  The caller allocates the
+ * pool with this size.  Host only.  0 on unsupported parameters. */
+size_t spark_pool_bytes(const spark_params *p);
+
 /* Bytes the method itself has to read per token and KV head in one decode step:
  * kept key values + mask + mu_pruned + the dense value row, or with value-channel pruning the
  * kept value entries + their mask (the roofline numerator).  Host only. */

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "SPARK_OK", 1: "SPARK_ERR_NULL", 2: "SPARK_ERR_BAD_SHAPE", 3:
                 7: "SPARK_ERR_DEVICE_TIMEOUT"}
 SPARK_F32, SPARK_BF16 = 0, 1
 _DTYPE_CODE = {torch.float32: SPARK_F32, torch.bfloat16: SPARK_BF16}
-EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes",
+EXPORTS = ["spark_version", "spark_last_launch_count", "spark_keep_count", "spark_page_bytes", "spark_pool_bytes",
            "spark_algorithmic_bytes_per_token", "spark_workspace_bytes", "spark_workspace_init",
            "spark_compress", "spark_append", "spark_append_block", "spark_merge_attn", "spark_decode_attn", "spark_decode_attn_host", "spark_decode_attn_noalloc", "spark_unpack_pages",
            "spark_unpack_value_masks", "spark_unpack_stats", "spark_group_keep", "spark_read_status"]
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.spark_keep_count.argtypes = [i32, ctypes.c_double]
         L.spark_page_bytes.restype = sz
         L.spark_page_bytes.argtypes = [P]
+        L.spark_pool_bytes.restype = sz
+        L.spark_pool_bytes.argtypes = [P]
         L.spark_algorithmic_bytes_per_token.restype = sz
         L.spark_algorithmic_bytes_per_token.argtypes = [P]
         L.spark_workspace_bytes.restype = i32
@@ -158,6 +160,10 @@ def spark_group_keep(head_dim: int, group_prune) -> int:
 
 def spark_page_bytes(p: spark_params) -> int:
     return int(lib().spark_page_bytes(ctypes.byref(p)))
+
+
+def spark_pool_bytes(p: spark_params) -> int:
+    return int(lib().spark_pool_bytes(ctypes.byref(p)))
 
 
 def spark_algorithmic_bytes_per_token(p: spark_params) -> int:

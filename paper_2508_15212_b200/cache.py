@@ -51,7 +51,7 @@ class SparkCache:
                                     group_prune=group_prune, recovery=recovery, seed=seed)
         self.page_bytes = B.spark_page_bytes(self.params)
         assert self.page_bytes > 0
-        self.pages = pages if pages is not None else self._alloc("pages", n_pool_pages * self.page_bytes, zero=True)
+        self.pages = pages if pages is not None else self._alloc("pages", B.spark_pool_bytes(self.params), zero=True)
         self.qnorm = self._alloc("qnorm", batch * n_kv_heads * 128 * 4).view(torch.float32).view(batch, n_kv_heads, 128)
         self.packed_lens = self._alloc("packed_lens", batch * 4, zero=True).view(torch.int32)
         self.kept_tokens = (self._alloc("kept_tokens", batch * n_kv_heads * token_budget * 4).view(torch.int32)

@@ -85,6 +85,15 @@ size_t spark_page_bytes(const spark_params* p)
     return static_cast<size_t>(make_layout(*p).page_bytes);
 }
 
+size_t spark_pool_bytes(const spark_params* p)
+{
+    const size_t page = spark_page_bytes(p);
+    if (!page || p->n_pool_pages < 1) return 0;
+    const PageLayout L = make_layout(*p);
+    if (!L.ragged) return page * static_cast<size_t>(p->n_pool_pages);
+    return static_cast<size_t>(rows_offset(p->n_pool_pages, L.page_bytes)) + static_cast<size_t>(p->n_pool_pages) * sizeof(int32_t);
+}
+
 size_t spark_algorithmic_bytes_per_token(const spark_params* p)
 {
     if (!p || p->keep < 1 || p->keep > p->head_dim || p->keep_v < 0 || p->keep_v > p->head_dim) return 0;

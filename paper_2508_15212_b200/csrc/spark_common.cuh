@@ -34,6 +34,8 @@ constexpr int kWorkspaceHeader = 256;
 //          a token = its s-th kept value channel), followed by
 //   vmask: [16][4] uint32 (pruned values only), bit (j % 32) of word (j / 32) set <=> value channel j kept
 struct PageLayout {
+    int vals_off;    // start of the kept key values (0, or behind everything else when `ragged`)
+    int ragged;      // SparK-p pages: the slot rows come last and a per-page row count says how many are in use
     int esize;       // bytes per element (2 bf16, 4 fp32)
     int keep;        // T
     int keep_v;      // T_v (128: dense value rows)
@@ -49,20 +51,36 @@ struct PageLayout {
 // spark_params.keep_v -> T_v (0 and 128 both mean dense value rows)
 __host__ __device__ inline int value_keep(int keep_v) { return (keep_v <= 0 || keep_v >= kHeadDim) ? kHeadDim : keep_v; }
 
-__host__ __device__ inline PageLayout make_layout(int dtype, int keep, int keep_v, int recovery)
+// With SparK-p the number of kept channels varies per token, so a page's slot rows are only used up to the
+// largest count among its 16 tokens.  Such pages are laid out with the slot rows LAST, and a row count per
+// pool page (int32, in a side array behind the pages of the pool) tells the decode step how many bytes of the
+// page to copy: mask | mu | (stats) | values | the first `rows` slot rows.
+__host__ __device__ inline PageLayout make_layout(int dtype, int keep, int keep_v, int recovery, int ragged = 0)
 {
     PageLayout L;
     L.esize = (dtype == SPARK_BF16) ? 2 : 4;
     L.keep = keep;
     L.keep_v = value_keep(keep_v);
-    L.mask_off = keep * kPageTokens * L.esize;
+    L.ragged = ragged;
+    L.vals_off = 0;
+    L.mask_off = ragged ? 0 : keep * kPageTokens * L.esize;
     L.mu_off = L.mask_off + kPageTokens * 16;
     L.stats_off = L.mu_off + kPageTokens * 4;
     L.recovery = recovery;
     L.v_off = L.stats_off + (recovery != SPARK_RECOVER_DEGENERATE ? 2 * kPageTokens * 4 : 0);
     L.vmask_off = L.v_off + L.keep_v * kPageTokens * L.esize;
     L.page_bytes = L.vmask_off + (L.keep_v < kHeadDim ? kPageTokens * 16 : 0);
+    if (ragged) {
+        L.vals_off = L.page_bytes;
+        L.page_bytes += keep * kPageTokens * L.esize;
+    }
     return L;
+}
+
+// the per-page row counts of a ragged pool: an int32 per pool page behind the pages (256-byte aligned)
+__host__ __device__ inline int64_t rows_offset(int64_t n_pool_pages, int page_bytes)
+{
+    return (n_pool_pages * page_bytes + 255) / 256 * 256;
 }
 
 // byte offset of kept slot s of token p inside the vals section
@@ -115,7 +133,10 @@ spark_status launch_unpack(const spark_params& p, const void* pages, const int32
                            int32_t max_blocks, const int32_t* packed_lens, int32_t max_tokens,
                            uint32_t* mask, float* mu, void* vals, void* v, uint32_t* vmask, float* mu_all,
                            float* sigma_all, cudaStream_t stream);
-inline PageLayout make_layout(const spark_params& p) { return make_layout(p.dtype, p.keep, p.keep_v, p.recovery); }
+inline PageLayout make_layout(const spark_params& p)
+{
+    return make_layout(p.dtype, p.keep, p.keep_v, p.recovery, p.select == SPARK_SELECT_TOP_P ? 1 : 0);
+}
 int group_keep(int head_dim, int n_groups, const float* prune);
 
 spark_status launch_decode(const spark_params& p, const void* q, const void* pages,

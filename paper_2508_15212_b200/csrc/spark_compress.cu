@@ -212,8 +212,8 @@ __device__ __forceinline__ int select_by_rank(const unsigned (&key)[4], int lane
     return n_kept;
 }
 
-template <bool kBf16>
-__device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, int mask_off, int mu_off,
+template <bool kBf16, bool kRank>
+__device__ __forceinline__ int pack_token(unsigned char* image, int vals_off, int mask_off, int mu_off,
                                            int p, int T, int lane,
                                            const float (&a)[4], const float (&kf)[4], const unsigned (&raw)[4],
                                            double inv_pruned = 0.0, const SelectArgs* sel = nullptr, int stats_off = -1)
@@ -228,7 +228,7 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
     }
     bool kept[4];
     int n_kept = T;
-    if (sel && sel->select != SPARK_SELECT_FIXED) n_kept = select_by_rank(key, lane, *sel, T, kept);   // warp-uniform
+    if (kRank) n_kept = select_by_rank(key, lane, *sel, T, kept);     // a ratio-free rule (keys only)
     else select_top_t(key, T, lane, kept);
     // slot of each kept channel = kept channels below it
     int slot = 0;
@@ -256,18 +256,18 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
     word |= __shfl_xor_sync(kFullMask, word, 4);
     if ((lane & 7) == 0)
         reinterpret_cast<unsigned*>(image + mask_off)[p * kMaskWords + (lane >> 3)] = word;
-    if (mu_off < 0) return;                                   // warp-uniform
+    if (mu_off < 0) return n_kept;                            // warp-uniform
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) pruned += __shfl_xor_sync(kFullMask, pruned, o);
     if (lane == 0) {
         float mu;
-        if (sel && sel->select != SPARK_SELECT_FIXED)
+        if (kRank)
             mu = n_kept < kHeadDim ? static_cast<float>(pruned / static_cast<double>(kHeadDim - n_kept)) : 0.f;
         else
             mu = static_cast<float>(pruned * inv_pruned);
         reinterpret_cast<float*>(image + mu_off)[p] = mu;
     }
-    if (stats_off < 0) return;                                // warp-uniform
+    if (stats_off < 0) return n_kept;                         // warp-uniform
     // all-channel mean and population deviation of the token's saliencies (sampled recovery)
     double s1 = (static_cast<double>(w[0]) + static_cast<double>(w[1])) + (static_cast<double>(w[2]) + static_cast<double>(w[3]));
 #pragma unroll
@@ -282,13 +282,14 @@ __device__ __forceinline__ void pack_token(unsigned char* image, int vals_off, i
         reinterpret_cast<float*>(image + stats_off)[p] = static_cast<float>(mean);
         reinterpret_cast<float*>(image + stats_off)[kPageTokens + p] = static_cast<float>(sqrt(s2 / static_cast<double>(kHeadDim)));
     }
+    return n_kept;
 }
 
 // Key entries and value entries of one token row into the page image.  A lane owns channels 4*lane ..
 // 4*lane+3; `row` is the element offset of its first channel in k and v.  `inv_pruned` = 1 / (D - T)
 // (0 when T = D), computed once on the host.
-template <bool kBf16>
-__device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLayout& L, int p, int lane,
+template <bool kBf16, bool kRank>
+__device__ __forceinline__ int pack_token_kv(unsigned char* image, const PageLayout& L, int p, int lane,
                                               const float (&a)[4], const void* k, const void* v, int64_t row,
                                               double inv_pruned, const SelectArgs& sel)
 {
@@ -319,10 +320,10 @@ __device__ __forceinline__ void pack_token_kv(unsigned char* image, const PageLa
 #pragma unroll
         for (int i = 0; i < 4; ++i) vf[i] = __uint_as_float(kBf16 ? vraw[i] << 16 : vraw[i]);
         const float one[4] = {1.f, 1.f, 1.f, 1.f};
-        pack_token<kBf16>(image, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
+        pack_token<kBf16, false>(image, L.v_off, L.vmask_off, -1, p, L.keep_v, lane, one, vf, vraw);
     }
-    pack_token<kBf16>(image, 0, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned, &sel,
-                      L.recovery != SPARK_RECOVER_DEGENERATE ? L.stats_off : -1);
+    return pack_token<kBf16, kRank>(image, L.vals_off, L.mask_off, L.mu_off, p, L.keep, lane, a, kf, kraw, inv_pruned, &sel,
+                             L.recovery != SPARK_RECOVER_DEGENERATE ? L.stats_off : -1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -353,7 +354,7 @@ struct CompressArgs {
     int* status;
 };
 
-template <typename E>
+template <typename E, bool kRank>
 __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
 {
     extern __shared__ __align__(16) unsigned char image[];
@@ -364,6 +365,8 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     const PageLayout L = A.L;
     constexpr bool kBf16 = (sizeof(E) == 2);
 
+    __shared__ int rows_used;
+    if (threadIdx.x == 0) rows_used = 0;
     for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
         reinterpret_cast<uint4*>(image)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
@@ -378,7 +381,8 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
             ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
         const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
                             static_cast<int64_t>(src_t) * A.st + lane * 4;
-        pack_token_kv<kBf16>(image, L, p, lane, a, A.k, A.v, row, A.inv_pruned, A.sel);
+        const int n_kept = pack_token_kv<kBf16, kRank>(image, L, p, lane, a, A.k, A.v, row, A.inv_pruned, A.sel);
+        if (kRank && L.ragged && lane == 0) atomicMax(&rows_used, n_kept);
     }
     __syncthreads();
 
@@ -391,6 +395,8 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
     uint4* dst = reinterpret_cast<uint4*>(A.pages + page_id * L.page_bytes);
     for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
         dst[i] = reinterpret_cast<const uint4*>(image)[i];
+    if (kRank && L.ragged && threadIdx.x == 0)
+        reinterpret_cast<int*>(A.pages + rows_offset(A.n_pool_pages, L.page_bytes))[page_id] = rows_used;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -414,7 +420,7 @@ struct AppendArgs {
     int* status;
 };
 
-template <typename E>
+template <typename E, bool kRank>
 __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
 {
     constexpr bool kBf16 = (sizeof(E) == 2);
@@ -433,14 +439,17 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
         return;
     }
     unsigned char* page = A.pages + page_id * L.page_bytes;
+    int* rows = L.ragged ? reinterpret_cast<int*>(A.pages + rows_offset(A.n_pool_pages, L.page_bytes)) + page_id : nullptr;
     if (p == 0) {                                             // first token of a page: clear it
         for (int i = lane; i < L.page_bytes / 16; i += 32) reinterpret_cast<uint4*>(page)[i] = make_uint4(0, 0, 0, 0);
+        if (rows && lane == 0) *rows = 0;
         __syncwarp();
     }
     const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
     const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
-    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+    const int n_kept = pack_token_kv<kBf16, kRank>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+    if (rows && lane == 0) atomicMax(rows, n_kept);
 }
 
 __global__ void append_advance_kernel(AppendArgs A)
@@ -475,9 +484,11 @@ __global__ void __launch_bounds__(32) append_block_clear_kernel(AppendBlockArgs 
     }
     uint4* page = reinterpret_cast<uint4*>(A.pages + page_id * A.L.page_bytes);
     for (int i = lane; i < A.L.page_bytes / 16; i += 32) page[i] = make_uint4(0, 0, 0, 0);
+    if (A.L.ragged && lane == 0)
+        reinterpret_cast<int*>(A.pages + rows_offset(A.n_pool_pages, A.L.page_bytes))[page_id] = 0;
 }
 
-template <typename E>
+template <typename E, bool kRank>
 __global__ void __launch_bounds__(32) append_block_token_kernel(AppendBlockArgs B_)
 {
     constexpr bool kBf16 = (sizeof(E) == 2);
@@ -502,7 +513,9 @@ __global__ void __launch_bounds__(32) append_block_token_kernel(AppendBlockArgs 
     const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
     const float a[4] = {a4.x, a4.y, a4.z, a4.w};
     const int64_t row = ((static_cast<int64_t>(b) * A.Hkv + h) * B_.n_new + tok) * kHeadDim + lane * 4;
-    pack_token_kv<kBf16>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+    const int n_kept = pack_token_kv<kBf16, kRank>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+    if (L.ragged && lane == 0)
+        atomicMax(reinterpret_cast<int*>(A.pages + rows_offset(A.n_pool_pages, L.page_bytes)) + page_id, n_kept);
 }
 
 __global__ void append_block_advance_kernel(AppendBlockArgs B_)
@@ -547,8 +560,14 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     A.sel = make_select(p);
     A.status = static_cast<int*>(workspace);
     const dim3 grid(p.n_kv_heads, p.batch);
-    if (p.dtype == SPARK_BF16) append_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(A);
-    else append_token_kernel<float><<<grid, 32, 0, stream>>>(A);
+    const bool rank = p.select != SPARK_SELECT_FIXED;
+    if (p.dtype == SPARK_BF16) {
+        if (rank) append_token_kernel<__nv_bfloat16, true><<<grid, 32, 0, stream>>>(A);
+        else append_token_kernel<__nv_bfloat16, false><<<grid, 32, 0, stream>>>(A);
+    } else {
+        if (rank) append_token_kernel<float, true><<<grid, 32, 0, stream>>>(A);
+        else append_token_kernel<float, false><<<grid, 32, 0, stream>>>(A);
+    }
     append_advance_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(A);
     *launches += 2;
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
@@ -571,8 +590,14 @@ spark_status launch_append_block(const spark_params& p, const void* k_new, const
     const int fresh = (n_new + kPageTokens - 1) / kPageTokens + 1;       // pages that can start inside the new tokens
     append_block_clear_kernel<<<dim3(p.n_kv_heads, p.batch, fresh), 32, 0, stream>>>(Bk);
     const dim3 grid(p.n_kv_heads, p.batch, n_new);
-    if (p.dtype == SPARK_BF16) append_block_token_kernel<__nv_bfloat16><<<grid, 32, 0, stream>>>(Bk);
-    else append_block_token_kernel<float><<<grid, 32, 0, stream>>>(Bk);
+    const bool rank = p.select != SPARK_SELECT_FIXED;
+    if (p.dtype == SPARK_BF16) {
+        if (rank) append_block_token_kernel<__nv_bfloat16, true><<<grid, 32, 0, stream>>>(Bk);
+        else append_block_token_kernel<__nv_bfloat16, false><<<grid, 32, 0, stream>>>(Bk);
+    } else {
+        if (rank) append_block_token_kernel<float, true><<<grid, 32, 0, stream>>>(Bk);
+        else append_block_token_kernel<float, false><<<grid, 32, 0, stream>>>(Bk);
+    }
     append_block_advance_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(Bk);
     *launches += 3;
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
@@ -677,10 +702,10 @@ __global__ void __launch_bounds__(128) unpack_pages_kernel(UnpackArgs A)
             const int64_t o = (row0 + p) * T + s;
             if (L.esize == 2)
                 static_cast<unsigned short*>(A.vals)[o] =
-                    live ? *reinterpret_cast<const unsigned short*>(page + val_offset(2, p, s)) : 0;
+                    live ? *reinterpret_cast<const unsigned short*>(page + L.vals_off + val_offset(2, p, s)) : 0;
             else
                 static_cast<unsigned*>(A.vals)[o] =
-                    live ? *reinterpret_cast<const unsigned*>(page + val_offset(4, p, s)) : 0u;
+                    live ? *reinterpret_cast<const unsigned*>(page + L.vals_off + val_offset(4, p, s)) : 0u;
         }
     if (A.vmask)                                                  // all ones for dense value rows
         for (int i = threadIdx.x; i < kPageTokens * kMaskWords; i += blockDim.x) {
@@ -758,10 +783,14 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
     A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
     A.sel = make_select(p);
     const dim3 grid(n_blocks, p.n_kv_heads, p.batch);
-    if (p.dtype == SPARK_BF16)
-        compress_pages_kernel<__nv_bfloat16><<<grid, 256, A.L.page_bytes, stream>>>(A);
-    else
-        compress_pages_kernel<float><<<grid, 256, A.L.page_bytes, stream>>>(A);
+    const bool rank = p.select != SPARK_SELECT_FIXED;      // a ratio-free rule: the kernels with the rank sort
+    if (p.dtype == SPARK_BF16) {
+        if (rank) compress_pages_kernel<__nv_bfloat16, true><<<grid, 256, A.L.page_bytes, stream>>>(A);
+        else compress_pages_kernel<__nv_bfloat16, false><<<grid, 256, A.L.page_bytes, stream>>>(A);
+    } else {
+        if (rank) compress_pages_kernel<float, true><<<grid, 256, A.L.page_bytes, stream>>>(A);
+        else compress_pages_kernel<float, false><<<grid, 256, A.L.page_bytes, stream>>>(A);
+    }
     ++*launches;
     if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
     return SPARK_OK;

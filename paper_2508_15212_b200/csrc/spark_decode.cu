@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
                     const unsigned words[4] = {mk.x, mk.y, mk.z, mk.w};
                     // kept slot s of token p (see val_offset): fp32 rows hold token p at element p, bf16 rows at
                     // element (p & 7) * 2 + (p >> 3); rows are 16 elements apart
-                    const unsigned char* vp = page + (kBf16 ? ((p & 7) * 2 + (p >> 3)) * 2 : p * 4);
+                    const unsigned char* vp = page + L.vals_off + (kBf16 ? ((p & 7) * 2 + (p >> 3)) * 2 : p * 4);
                     constexpr int kRowBytes = kPageTokens * static_cast<int>(sizeof(E));
                     float a[G];
 #pragma unroll
@@ -416,6 +416,7 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.nslots = 0; A.slot_stride = 0; A.pps = 1; A.prefix_off = 0; A.ring_off = 0;
     A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
     A.seed = p.seed;
+    A.page_rows = A.L.ragged ? reinterpret_cast<const int*>(A.pages + rows_offset(p.n_pool_pages, A.L.page_bytes)) : nullptr;
     const spark_status st = (p.dtype != SPARK_BF16) ? launch_decode_f32(G, A, dev, info, stream)
                             : (p.recovery != SPARK_RECOVER_DEGENERATE) ? launch_decode_bf16_sampled(G, A, dev, info, stream)
                                                                        : launch_decode_bf16(G, A, dev, info, stream);

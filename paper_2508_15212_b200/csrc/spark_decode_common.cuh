@@ -44,6 +44,7 @@ struct DecodeArgs {
     int ring_off;                            // shared-memory offset of the ring (behind the prefix)
     int overlap;                             // launched as a programmatic dependent of the preceding kernel
     unsigned seed;                           // sampled recovery: seed of the per-entry draws
+    const int* page_rows;                    // ragged pages: slot rows in use per pool page (else null: whole pages)
 };
 
 // control block at the start of dynamic shared memory
@@ -402,10 +403,19 @@ __device__ __forceinline__ void unit_parts(const Plan& pl, int unit_start, int u
 // behind the wait), then the warp polls: a lane whose slot has been released by the consumers arms
 // the slot's barrier and issues its page copies at once.  Polling is bounded; on expiry the CTA-wide
 // abort flag is set and the lanes wait (bounded) for their own copies in flight before returning.
-__device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctrl& C, int g, int c1, bool active,
-                                                  int& id0, int& id1)
+// bytes of page `id` to bring in: everything, or (ragged pages) up to the last slot row in use
+__device__ __forceinline__ unsigned page_copy_bytes(const DecodeArgs& A, int id)
 {
-    id0 = -1; id1 = -1;
+    if (!A.page_rows) return static_cast<unsigned>(A.L.page_bytes);
+    int rows = A.page_rows[id];
+    rows = rows < 0 ? 0 : (rows > A.L.keep ? A.L.keep : rows);
+    return static_cast<unsigned>(A.L.vals_off + rows * kPageTokens * A.L.esize);
+}
+
+__device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctrl& C, int g, int c1, bool active,
+                                                  int& id0, int& id1, unsigned& n0, unsigned& n1)
+{
+    id0 = -1; id1 = -1; n0 = 0; n1 = 0;
     if (!active) return;
     const Segment s = locate(C.prefix, A.B, A.Hkv, g, c1);
     const int64_t row = (static_cast<int64_t>(s.b) * A.Hkv + s.h) * A.max_blocks;
@@ -416,9 +426,11 @@ __device__ __forceinline__ void producer_page_ids(const DecodeArgs& A, const Ctr
         if (2 * s.i0 + 1 < (len + kPageTokens - 1) / kPageTokens) {
             id1 = bt ? bt[2 * s.i0 + 1] : static_cast<int>(row + 2 * s.i0 + 1);
             if (id1 < 0 || id1 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id1 = 0; }
+            n1 = page_copy_bytes(A, id1);
         }
     }
     if (id0 < 0 || id0 >= A.n_pool_pages) { record_error(A.status, SPARK_ERR_DEVICE_BOUNDS); id0 = 0; }
+    n0 = page_copy_bytes(A, id0);
 }
 
 __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C, unsigned char* ring,
@@ -434,32 +446,32 @@ __device__ __forceinline__ void producer_loop(const DecodeArgs& A, const Ctrl& C
     bool live = true;
     int last_round = -1;                                   // last revolution in which this lane issued
     int id0, id1;
-    producer_page_ids(A, C, c0 + lane, c1, owner && lane < n_total, id0, id1);
+    unsigned n0, n1;                                       // bytes to copy of the two pages
+    producer_page_ids(A, C, c0 + lane, c1, owner && lane < n_total, id0, id1, n0, n1);
     for (int round = 0; round * NS < n_total; ++round) {
         const int n = round * NS + lane;
         bool pending = owner && n < n_total;
         const int cur0 = id0, cur1 = id1;
+        const unsigned b0 = n0, b1 = n1;
         // next revolution's ids: the lookup waits for its block-table loads, so it runs before the poll
         // (hidden behind the wait for free slots) except in the first revolution, where every slot is
         // free and the copies go out first
-        if (round > 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
+        if (round > 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1, n0, n1);
         WaitClock wc;
         while (__any_sync(kFull, pending)) {
             if (pending && (round == 0 || mbar_try_wait(empty, (round - 1) & 1))) {
-                const unsigned bytes = L.page_bytes * (cur1 >= 0 ? 2u : 1u);
                 C.seq[lane] = round + 1;
-                mbar_expect_tx(full, bytes);
-                bulk_g2s(dst, A.pages + static_cast<int64_t>(cur0) * L.page_bytes, L.page_bytes, full, policy);
+                mbar_expect_tx(full, b0 + (cur1 >= 0 ? b1 : 0u));
+                bulk_g2s(dst, A.pages + static_cast<int64_t>(cur0) * L.page_bytes, b0, full, policy);
                 if (cur1 >= 0)
-                    bulk_g2s(dst + L.page_bytes, A.pages + static_cast<int64_t>(cur1) * L.page_bytes,
-                             L.page_bytes, full, policy);
+                    bulk_g2s(dst + L.page_bytes, A.pages + static_cast<int64_t>(cur1) * L.page_bytes, b1, full, policy);
                 last_round = round;
                 pending = false;
             }
             if (wc.expired() || *C.abort_flag) { live = false; break; }
         }
         if (!live) break;
-        if (round == 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1);
+        if (round == 0) producer_page_ids(A, C, c0 + n + NS, c1, owner && n + NS < n_total, id0, id1, n0, n1);
     }
     if (!live) {
         if (lane == 0) { *C.abort_flag = 1; record_error(A.status, SPARK_ERR_DEVICE_TIMEOUT); }

@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
                     if (c >= 1) x += t;
                     t = __shfl_up_sync(kFull, x, 2, 4);
                     if (c >= 2) x += t;
-                    vaddr[j] = page + (r * 2 + j) * 2 + (x - cnt) * 32;      // see val_offset: token r + 8j
+                    vaddr[j] = page + L.vals_off + (r * 2 + j) * 2 + (x - cnt) * 32;      // see val_offset: token r + 8j
                     vaddr_hi[j] = vaddr[j] + __popc(w[j] & 0xffffu) * 32;    // upper half of the word walks on its own
                 }
 #pragma unroll

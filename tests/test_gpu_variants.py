@@ -68,6 +68,16 @@ def check_selection(wl, cap, *, top_p=None, group_prune=None, block_table=None, 
         t = int(rng.integers(lens[b]))
         n = int(ref["count"][b, h, t])
         assert np.array_equal(vals[b, h, t, :n], kk[b, h, t][bits[b, h, t]]) and not vals[b, h, t, n:].any()
+    if top_p is not None and block_table is None:
+        # SparK-p pools carry, behind the pages, how many slot rows of each page are in use: the largest kept
+        # count among the page's live tokens (the decode step copies only that much of a page)
+        n_pages, pb = cache.params.n_pool_pages, cache.page_bytes
+        off = (n_pages * pb + 255) // 256 * 256
+        assert cache.pages.numel() == B.spark_pool_bytes(cache.params) == off + 4 * n_pages
+        rows = cache.pages[off:off + 4 * n_pages].view(torch.int32).cpu().numpy().reshape(Bn, Hkv, cache.table_blocks)
+        cnt = np.zeros((Bn, Hkv, cache.table_blocks * 16), np.int32)
+        cnt[:, :, :S] = ref["count"]
+        assert np.array_equal(rows, cnt.reshape(Bn, Hkv, cache.table_blocks, 16).max(axis=-1))
     out_ref, lse_ref = oracle.decode_attn(wl_cpu.q, wl_cpu.k, wl_cpu.v, wl_cpu.seq_lens, ref["mask"], ref["mu"], a)
     lse = cache.alloc_lse()
     out = cache.decode(wl.q, lse=lse)
