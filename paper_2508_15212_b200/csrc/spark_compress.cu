@@ -400,6 +400,257 @@ __global__ void __launch_bounds__(256) compress_pages_kernel(CompressArgs A)
 }
 
 // ------------------------------------------------------------------------------------------------
+// Fixed-T pages, four tokens per warp.  Most of what the selection costs per token is warp-wide
+// bookkeeping (reductions, votes, loop control) that serves one token when a warp owns one token.  Here a
+// token belongs to EIGHT lanes (16 channels per lane), a warp carries four tokens through the same
+// instructions, and the radix descent compares two keys per instruction while it works on the keys' upper
+// 16 bits (the bf16 image of a non-negative float orders like the float): `set.ge.u32.bf16x2` yields a
+// 0xFFFF / 0 half-word mask per key, eight such masks are folded into one word with one logic op each and
+// counted with one population count.  Below bit 16 the descent continues on the full keys.  The result is
+// the same exact top-T set, with ties to the lower channel, as select_top_t.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int group8_sum(int v)              // (a masked hardware reduction measured slower)
+{
+    v += __shfl_xor_sync(kFullMask, v, 1);
+    v += __shfl_xor_sync(kFullMask, v, 2);
+    v += __shfl_xor_sync(kFullMask, v, 4);
+    return v;
+}
+__device__ __forceinline__ double group8_sum(double v)
+{
+    v += __shfl_xor_sync(kFullMask, v, 1);
+    v += __shfl_xor_sync(kFullMask, v, 2);
+    v += __shfl_xor_sync(kFullMask, v, 4);
+    return v;
+}
+__device__ __forceinline__ int group8_exclusive(int v, int l8)      // sum over the lower lanes of the group
+{
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+        const int y = __shfl_up_sync(kFullMask, x, o, 8);
+        if (l8 >= o) x += y;
+    }
+    return x - v;
+}
+// per half: 1.0 (bf16) where a >= b, else 0 -- on the half-precision pipe, so that counting the keys at or
+// above a candidate costs the integer pipe nothing
+__device__ __forceinline__ __nv_bfloat162 ge_one_bf16x2(unsigned a, unsigned b)
+{
+    return __hge2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+}
+
+// kept bits (bit i <=> the lane's channel i) of the exact top-T among the 128 keys of the lane's group
+__device__ __forceinline__ unsigned select_top_t16(const unsigned (&key)[16], int T, int l8)
+{
+    unsigned hk[8];                                              // upper halves of the keys, two per word
+#pragma unroll
+    for (int i = 0; i < 8; ++i) hk[i] = (key[2 * i] >> 16) | (key[2 * i + 1] & 0xffff0000u);
+    // bits in which the group's keys differ: from the upper halves, and from the full keys only when the
+    // upper halves all agree
+    unsigned o = hk[0], n = hk[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) { o |= hk[i]; n &= hk[i]; }
+    o |= o << 16; n &= n << 16;                                  // fold the two keys of a word into the upper half
+#pragma unroll
+    for (int d = 1; d < 8; d <<= 1) {
+        o |= __shfl_xor_sync(kFullMask, o, d);
+        n &= __shfl_xor_sync(kFullMask, n, d);
+    }
+    o &= 0xffff0000u; n &= 0xffff0000u;
+    if (__any_sync(kFullMask, o == n)) {                         // rare: some group's keys share their upper halves
+        unsigned o2 = key[0], n2 = key[0];
+#pragma unroll
+        for (int i = 1; i < 16; ++i) { o2 |= key[i]; n2 &= key[i]; }
+#pragma unroll
+        for (int d = 1; d < 8; d <<= 1) {
+            o2 |= __shfl_xor_sync(kFullMask, o2, d);
+            n2 &= __shfl_xor_sync(kFullMask, n2, d);
+        }
+        o = o2; n = n2;
+    } else {
+        o |= 0xffffu;                                            // lower halves: treated as differing everywhere
+    }
+    const unsigned diff = o ^ n;
+    const int top = diff ? (31 - __clz(diff)) : -1;              // highest bit in which the group's keys differ
+    unsigned thr = (top >= 0) ? (n & ~((2u << top) - 1u)) : n;   // common leading bits
+    bool done = top < 0, exact = false;
+    const int start = __reduce_max_sync(kFullMask, top);
+    int bit = start;
+    for (; bit >= 16; --bit) {
+        if (__all_sync(kFullMask, done)) break;
+        const bool act = !done && bit <= top;
+        const unsigned cand = thr | (1u << bit);
+        const unsigned c2 = (cand >> 16) * 0x00010001u;
+        __nv_bfloat162 g[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) g[i] = ge_one_bf16x2(hk[i], c2);
+        const __nv_bfloat162 acc = __hadd2(__hadd2(__hadd2(g[0], g[1]), __hadd2(g[2], g[3])),
+                                           __hadd2(__hadd2(g[4], g[5]), __hadd2(g[6], g[7])));   // counts <= 8: exact in bf16
+        const int cnt = group8_sum(static_cast<int>(__low2float(acc) + __high2float(acc)));
+        if (act && cnt >= T) thr = cand;
+        if (act && cnt == T) { exact = true; done = true; }
+    }
+    for (bit = bit > 15 ? 15 : bit; bit >= 0; --bit) {
+        if (__all_sync(kFullMask, done)) break;
+        const bool act = !done && bit <= top;
+        const unsigned cand = thr | (1u << bit);
+        int mine = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) mine += (key[i] >= cand) ? 1 : 0;
+        const int cnt = group8_sum(mine);
+        if (act && cnt >= T) thr = cand;
+        if (act && cnt == T) { exact = true; done = true; }
+    }
+    unsigned kept = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) kept |= (key[i] >= thr) ? (1u << i) : 0u;
+    if (__any_sync(kFullMask, !exact)) {
+        // not an exact split: thr is the T-th largest key and the keys equal to it are admitted in ascending
+        // channel order (lanes ascending, channels inside a lane ascending) until T channels are kept
+        int n_gt = 0, n_eq = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            n_gt += (key[i] > thr) ? 1 : 0;
+            n_eq += (key[i] == thr) ? 1 : 0;
+        }
+        const int need_eq = T - group8_sum(n_gt);
+        int rank = group8_exclusive(n_eq, l8);
+        if (!exact) {
+            kept = 0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const bool eq = key[i] == thr;
+                if (key[i] > thr || (eq && rank < need_eq)) kept |= 1u << i;
+                rank += eq ? 1 : 0;
+            }
+        }
+    }
+    return kept;
+}
+
+// One token of one KV head handled by the eight lanes of a group: saliency, selection, and the token's
+// entries of the page image.  The lane owns channels 16*l8 .. 16*l8+15; `raw` holds their stored bit patterns
+// (two bf16 per word, or one fp32 per word).  Same outputs as pack_token.
+template <bool kBf16>
+__device__ __forceinline__ void pack_token16(unsigned char* image, int vals_off, int mask_off, int mu_off,
+                                             int stats_off, int p, int T, int l8, bool live,
+                                             const float* __restrict__ a, const unsigned* raw, double inv_pruned)
+{
+    unsigned key[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float kf = kBf16 ? __uint_as_float((i & 1) ? (raw[i >> 1] & 0xffff0000u) : (raw[i >> 1] << 16))
+                               : __uint_as_float(raw[i]);
+        key[i] = __float_as_uint(__fmul_rn(a ? a[i] : 1.f, fabsf(kf)));     // the one rounding that decides selection
+    }
+    const unsigned kept = select_top_t16(key, T, l8);
+    const int slot0 = group8_exclusive(__popc(kept), l8);
+    double pruned = 0.0, s1 = 0.0;
+    if (live) {
+        unsigned char* dst = image + vals_off + val_offset(kBf16 ? 2 : 4, p, slot0);
+        constexpr int kRow = kPageTokens * (kBf16 ? 2 : 4);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if ((kept >> i) & 1u) {
+                if (kBf16) *reinterpret_cast<unsigned short*>(dst) =
+                               static_cast<unsigned short>((i & 1) ? (raw[i >> 1] >> 16) : (raw[i >> 1] & 0xffffu));
+                else *reinterpret_cast<unsigned*>(dst) = raw[i];
+                dst += kRow;
+            } else {
+                pruned += static_cast<double>(__uint_as_float(key[i]));
+            }
+        }
+    }
+    const unsigned other = __shfl_xor_sync(kFullMask, kept, 1);
+    if (live && (l8 & 1) == 0)
+        reinterpret_cast<unsigned*>(image + mask_off)[p * kMaskWords + (l8 >> 1)] = kept | (other << 16);
+    if (mu_off < 0) return;                                   // warp-uniform
+    pruned = group8_sum(pruned);
+    if (live && l8 == 0) reinterpret_cast<float*>(image + mu_off)[p] = static_cast<float>(pruned * inv_pruned);
+    if (stats_off < 0) return;                                // warp-uniform
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s1 += static_cast<double>(__uint_as_float(key[i]));
+    const double mean = group8_sum(s1) / static_cast<double>(kHeadDim);
+    double s2 = 0.0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { const double d = static_cast<double>(__uint_as_float(key[i])) - mean; s2 += d * d; }
+    s2 = group8_sum(s2);
+    if (live && l8 == 0) {
+        reinterpret_cast<float*>(image + stats_off)[p] = static_cast<float>(mean);
+        reinterpret_cast<float*>(image + stats_off)[kPageTokens + p] = static_cast<float>(sqrt(s2 / static_cast<double>(kHeadDim)));
+    }
+}
+
+template <typename E>
+__global__ void __launch_bounds__(128, 8) compress_pages4_kernel(CompressArgs A)
+{
+    extern __shared__ __align__(16) unsigned char image[];
+    constexpr bool kBf16 = (sizeof(E) == 2);
+    constexpr int kWords = kBf16 ? 8 : 16;                     // 32-bit words of a lane's 16 channels
+    const int blk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int len = A.lens[b];
+    if (blk * kPageTokens >= len) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, l8 = lane & 7;
+    const int p = warp * 4 + (lane >> 3);                      // this group's token of the page
+    const PageLayout L = A.L;
+
+    for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(image)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    float a[16];
+    {
+        const float4* src = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim) + 4 * l8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = src[i];
+            a[4 * i] = f.x; a[4 * i + 1] = f.y; a[4 * i + 2] = f.z; a[4 * i + 3] = f.w;
+        }
+    }
+    const int t = blk * kPageTokens + p;
+    const bool live = t < len;
+    unsigned kraw[kWords], vraw[kWords];
+#pragma unroll
+    for (int i = 0; i < kWords; ++i) { kraw[i] = 0u; vraw[i] = 0u; }
+    if (live) {
+        const int src_t = A.gather ? A.gather[(static_cast<int64_t>(b) * A.Hkv + h) * A.gather_stride + t] : t;
+        const int64_t row = static_cast<int64_t>(b) * A.sb + static_cast<int64_t>(h) * A.sh +
+                            static_cast<int64_t>(src_t) * A.st + l8 * 16;
+        const uint4* ks = reinterpret_cast<const uint4*>(static_cast<const E*>(A.k) + row);
+        const uint4* vs = reinterpret_cast<const uint4*>(static_cast<const E*>(A.v) + row);
+#pragma unroll
+        for (int i = 0; i < kWords / 4; ++i) {
+            const uint4 kk = ks[i], vv = vs[i];
+            kraw[4 * i] = kk.x; kraw[4 * i + 1] = kk.y; kraw[4 * i + 2] = kk.z; kraw[4 * i + 3] = kk.w;
+            vraw[4 * i] = vv.x; vraw[4 * i + 1] = vv.y; vraw[4 * i + 2] = vv.z; vraw[4 * i + 3] = vv.w;
+        }
+        if (L.keep_v >= kHeadDim) {                        // dense value row: the lane's 16-byte chunks
+#pragma unroll
+            for (int i = 0; i < kWords / 4; ++i)
+                *reinterpret_cast<uint4*>(image + L.v_off + v_chunk_offset(kBf16 ? 2 : 4, p, (kWords / 4) * l8 + i)) =
+                    make_uint4(vraw[4 * i], vraw[4 * i + 1], vraw[4 * i + 2], vraw[4 * i + 3]);
+        }
+    }
+    if (L.keep_v < kHeadDim)                               // value-channel pruning: same selection on |V|
+        pack_token16<kBf16>(image, L.v_off, L.vmask_off, -1, -1, p, L.keep_v, l8, live, nullptr, vraw, 0.0);
+    pack_token16<kBf16>(image, L.vals_off, L.mask_off, L.mu_off,
+                        L.recovery != SPARK_RECOVER_DEGENERATE ? L.stats_off : -1, p, L.keep, l8, live, a, kraw,
+                        A.inv_pruned);
+    __syncthreads();
+
+    const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+    const int64_t page_id = A.block_table ? A.block_table[entry] : entry;     // no table: contiguous cache
+    if (page_id < 0 || page_id >= A.n_pool_pages) {
+        if (threadIdx.x == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(A.pages + page_id * L.page_bytes);
+    for (int i = threadIdx.x; i < L.page_bytes / 16; i += blockDim.x)
+        dst[i] = reinterpret_cast<const uint4*>(image)[i];
+}
+
+// ------------------------------------------------------------------------------------------------
 // Decode-time append: one new token per sequence is pruned with the sequence's prefill statistics
 // (qnorm) and written into the next token slot of its last page (a fresh page is zeroed first).
 // One warp per (sequence, KV head); a second one-thread-per-sequence kernel advances packed_lens.
@@ -786,10 +1037,10 @@ spark_status launch_compress(const spark_params& p, const void* q_win, const voi
     const bool rank = p.select != SPARK_SELECT_FIXED;      // a ratio-free rule: the kernels with the rank sort
     if (p.dtype == SPARK_BF16) {
         if (rank) compress_pages_kernel<__nv_bfloat16, true><<<grid, 256, A.L.page_bytes, stream>>>(A);
-        else compress_pages_kernel<__nv_bfloat16, false><<<grid, 256, A.L.page_bytes, stream>>>(A);
+        else compress_pages4_kernel<__nv_bfloat16><<<grid, 128, A.L.page_bytes, stream>>>(A);
     } else {
         if (rank) compress_pages_kernel<float, true><<<grid, 256, A.L.page_bytes, stream>>>(A);
-        else compress_pages_kernel<float, false><<<grid, 256, A.L.page_bytes, stream>>>(A);
+        else compress_pages4_kernel<float><<<grid, 128, A.L.page_bytes, stream>>>(A);
     }
     ++*launches;
     if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
