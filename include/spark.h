@@ -117,7 +117,13 @@ typedef enum {
      * only after that preceding kernel has completed.  Set it only when the preceding kernel does not
      * write the packed cache, the block table or packed_lens (a projection that produces q is fine).
      * Results are identical with and without the flag. */
-    SPARK_FLAG_OVERLAP_PREVIOUS = 1
+    SPARK_FLAG_OVERLAP_PREVIOUS = 1,
+    /* spark_decode_attn_host only.  q_host, out_host (and lse_host) are page-locked host memory that the device
+     * can address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel reads the query and
+     * writes the result across the bus itself, no staging copies are enqueued, and q_dev / out_dev / lse_dev
+     * may be NULL.  If the runtime cannot give a device address for one of them the call returns
+     * SPARK_ERR_BAD_SHAPE before anything is enqueued. */
+    SPARK_FLAG_HOST_MAPPED = 2
 } spark_flags;
 
 /* T = floor((1 - ratio) * head_dim): the paper's kept-channel count (Sec. "Problem
@@ -274,6 +280,7 @@ spark_status spark_decode_attn(const spark_params *p, const void *q,
  * of lse_dev to lse_host when both are given).  Nothing is synchronised: the results are in out_host once
  * the stream has reached this point.
  *
+ *   (With SPARK_FLAG_HOST_MAPPED the two copies are replaced by direct device access to the host buffers.)
  *   q_host             HOST [B][Hq][D], dtype as the cache; page-locked memory lets the copy run asynchronously
  *   q_dev              DEVICE staging for the query, same size, 16-byte aligned
  *   out_dev            DEVICE [B][Hq][D] fp32, 16-byte aligned;  out_host  HOST, same size

@@ -44,6 +44,7 @@ class spark_params(ctypes.Structure):
 
 
 SPARK_FLAG_OVERLAP_PREVIOUS = 1
+SPARK_FLAG_HOST_MAPPED = 2
 SPARK_SELECT_FIXED, SPARK_SELECT_TOP_P, SPARK_SELECT_GROUPS = 0, 1, 2
 SPARK_RECOVER_DEGENERATE, SPARK_RECOVER_GAUSSIAN, SPARK_RECOVER_EXPONENTIAL = 0, 1, 2
 

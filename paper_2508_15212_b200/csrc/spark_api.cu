@@ -30,7 +30,7 @@ spark_status spark::check_params(const spark_params* p)
     if (p->n_pool_pages < 1) return SPARK_ERR_BAD_SHAPE;
     if (p->token_budget < 0) return SPARK_ERR_BAD_SHAPE;
     if (!(p->qnorm_eps >= 0.f) || !(p->softmax_scale >= 0.f)) return SPARK_ERR_BAD_SHAPE;
-    if (p->flags & ~SPARK_FLAG_OVERLAP_PREVIOUS) return SPARK_ERR_BAD_SHAPE;
+    if (p->flags & ~(SPARK_FLAG_OVERLAP_PREVIOUS | SPARK_FLAG_HOST_MAPPED)) return SPARK_ERR_BAD_SHAPE;
     if (p->keep_v < 0 || p->keep_v > p->head_dim) return SPARK_ERR_BAD_SHAPE;
     if (p->select < SPARK_SELECT_FIXED || p->select > SPARK_SELECT_GROUPS) return SPARK_ERR_BAD_SHAPE;
     if (p->select == SPARK_SELECT_TOP_P && (!(p->top_p > 0.f) || !(p->top_p <= 1.f))) return SPARK_ERR_BAD_SHAPE;
@@ -243,7 +243,20 @@ spark_status spark_decode_attn_host(const spark_params* p, const void* q_host, v
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
-    if (!q_host || !q_dev || !out_dev || !out_host) return SPARK_ERR_NULL;
+    if (!q_host || !out_host) return SPARK_ERR_NULL;
+    if (p->flags & SPARK_FLAG_HOST_MAPPED) {
+        // the kernel addresses the page-locked host buffers itself: 8-24 KB cross the bus inside the step
+        void *dq = nullptr, *dout = nullptr, *dlse = nullptr;
+        if (cudaHostGetDevicePointer(&dq, const_cast<void*>(q_host), 0) != cudaSuccess ||
+            cudaHostGetDevicePointer(&dout, out_host, 0) != cudaSuccess ||
+            (lse_host && cudaHostGetDevicePointer(&dlse, lse_host, 0) != cudaSuccess)) {
+            cudaGetLastError();                            // clear the sticky-free error of the failed lookup
+            return SPARK_ERR_BAD_SHAPE;
+        }
+        return spark_decode_attn(p, dq, pages, block_table, max_blocks, packed_lens, qnorm, static_cast<float*>(dout),
+                                 static_cast<float*>(dlse), workspace, workspace_bytes, stream);
+    }
+    if (!q_dev || !out_dev) return SPARK_ERR_NULL;
     if ((lse_dev == nullptr) != (lse_host == nullptr)) return SPARK_ERR_NULL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t e = (p->dtype == SPARK_BF16) ? 2 : 4;

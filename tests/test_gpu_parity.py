@@ -408,6 +408,30 @@ def test_dense_tail_equals_the_oracle_with_appended_keys_left_dense(dtype, block
             assert np.allclose(lse.cpu().numpy(), ref_lse, rtol=0, atol=1e-3 if dtype == "bf16" else 2e-5)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_host_entry_point_staged_and_mapped_equal_the_device_call(dtype):
+    """spark_decode_attn_host: query and result in page-locked host memory, with staging copies or (flag) with the
+    kernel addressing the host buffers itself.  Both must give the device call's output bit for bit (which the
+    other tests tie to the oracle)."""
+    wl = make(dtype, 2, 8, 2, [700, 64], 8, 38, seed=170, sigma=1.0 if dtype == "bf16" else 0.5)
+    cache = SparkCache(batch=2, n_q_heads=8, n_kv_heads=2, window=8, keep=38, dtype=dtype, max_tokens=700)
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    ref = cache.decode(wl.q)
+    wl_cpu = wl.to("cpu")
+    a, c, o_ref, _ = oracle_side(wl_cpu, 38)
+    assert float(np.abs(ref.cpu().numpy() - o_ref).max()) <= TOL[dtype]
+    q_host = wl.q.cpu().pin_memory()
+    for flags in (0, B.SPARK_FLAG_HOST_MAPPED):
+        out_host = torch.full((2, 8, 128), float("nan"), dtype=torch.float32).pin_memory()
+        cache.params.flags = flags
+        call = cache.bind_decode_host(q_host, out_host)
+        call()
+        torch.cuda.synchronize()
+        assert torch.equal(out_host, ref.cpu()), f"flags={flags}"
+    cache.params.flags = 0
+    assert cache.status() == 0
+
+
 def test_merge_attn_handles_empty_sides():
     o = torch.randn(2, 4, 128, device="cuda")
     zero = torch.zeros_like(o)
