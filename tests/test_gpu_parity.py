@@ -126,6 +126,28 @@ def test_group_sizes_fp32(G, keep):
     check_case(wl, keep)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_selection_is_exact_on_subnormal_saliencies(dtype):
+    """Saliencies around 1e-39 (fp32 subnormals, whose upper 16 bits are bf16 subnormals): the selection must still
+    order them exactly -- nothing may be flushed to zero on the way to the kept set."""
+    wl = make(dtype, 2, 4, 2, [70, 33], 8, 64, seed=75, sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
+    tdt = wl.k.dtype
+    wl.k = (wl.k.float() * 2e-38).to(tdt)                       # the divisor's floor keeps a[j] ordinary: shrink K alone
+    wl_cpu = wl.to("cpu")
+    _, a = oracle.window_mean(wl_cpu.q_win, 2)
+    sal = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, 64, a, want_saliency=True)["saliency"]
+    live = sal[0, 0, :70]
+    assert 0 < live[live > 0].min() < 1.1754944e-38 and live.max() < 1e-36      # really in the subnormal range
+    for keep in (64, 25):
+        cache = SparkCache(batch=2, n_q_heads=4, n_kv_heads=2, window=8, keep=keep, dtype=dtype, max_tokens=70)
+        cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+        c = oracle.compress(wl_cpu.k, wl_cpu.seq_lens, keep, a)
+        u = cache.unpack(want_vals=False, want_v=False)
+        assert np.array_equal(cache.qnorm.cpu().numpy(), a)
+        assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c["mask"])
+        assert np.allclose(u["mu"].cpu().numpy(), c["mu"], rtol=1e-6, atol=0)
+
+
 def test_single_token_and_empty_sequence():
     wl = make("bf16", 3, 8, 2, [0, 1, 16], 4, 64, seed=70)
     check_case(wl, 64)
