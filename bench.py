@@ -535,8 +535,9 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     e2e_us = dist_utils.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") * 1e3 / e2e_steps
-    # the same call with SPARK_FLAG_HOST_MAPPED: the kernel reads q from and writes out to the pinned host
-    # buffers itself (no staging copies); reported beside the staged figure, which stays the e2e value
+    # the same call with SPARK_FLAG_HOST_MAPPED: the query travels inside the launch (or is read by the kernel)
+    # and the kernel writes the result into the pinned host buffer itself, no staging copies; reported beside
+    # the staged figure, which stays the e2e value
     for c in work.caches:
         c.params.flags = B.SPARK_FLAG_HOST_MAPPED
     for i in range(20):

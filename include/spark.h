@@ -119,10 +119,14 @@ typedef enum {
      * Results are identical with and without the flag. */
     SPARK_FLAG_OVERLAP_PREVIOUS = 1,
     /* spark_decode_attn_host only.  q_host, out_host (and lse_host) are page-locked host memory that the device
-     * can address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel reads the query and
-     * writes the result across the bus itself, no staging copies are enqueued, and q_dev / out_dev / lse_dev
-     * may be NULL.  If the runtime cannot give a device address for one of them the call returns
-     * SPARK_ERR_BAD_SHAPE before anything is enqueued. */
+     * can address (cudaHostAlloc / cudaHostRegister under unified addressing): the kernel writes the result
+     * across the bus itself, no staging copies are enqueued, and q_dev / out_dev / lse_dev may be NULL.  The
+     * query takes one of two routes.  bf16 storage, degenerate recovery, dense value rows and a query of at
+     * most 24 KB (B * Hq * 256 bytes): its bytes are read DURING THE CALL and travel to the GPU inside the
+     * kernel launch, so q_host must hold the query when the call is made (not merely when the stream gets
+     * there) and may be reused as soon as the call returns.  Otherwise the kernel reads q_host across the bus
+     * during the step (stream order, as without the flag).  If the runtime cannot give a device address for
+     * a buffer it needs, the call returns SPARK_ERR_BAD_SHAPE before anything is enqueued. */
     SPARK_FLAG_HOST_MAPPED = 2
 } spark_flags;
 

@@ -212,10 +212,11 @@ spark_status spark_merge_attn(int32_t batch, int32_t n_q_heads, int32_t head_dim
     return launch_merge_attn(batch * n_q_heads, out_a, lse_a, out_b, lse_b, out, lse, static_cast<cudaStream_t>(stream));
 }
 
-spark_status spark_decode_attn(const spark_params* p, const void* q, const void* pages,
-                               const int32_t* block_table, int32_t max_blocks,
-                               const int32_t* packed_lens, const float* qnorm, float* out, float* lse,
-                               void* workspace, size_t workspace_bytes, spark_stream_t stream)
+// spark_decode_attn proper; q_by_value: q is a host pointer whose bytes go into the launch (see launch_decode)
+static spark_status decode_attn(const spark_params* p, const void* q, const void* pages,
+                                const int32_t* block_table, int32_t max_blocks,
+                                const int32_t* packed_lens, const float* qnorm, float* out, float* lse,
+                                void* workspace, size_t workspace_bytes, spark_stream_t stream, bool q_by_value)
 {
     spark_status st = check_params(p);
     if (st != SPARK_OK) return st;
@@ -230,9 +231,18 @@ spark_status spark_decode_attn(const spark_params* p, const void* q, const void*
         return SPARK_ERR_WORKSPACE;
     int launches = 0;
     st = launch_decode(*p, q, pages, block_table, max_blocks, packed_lens, qnorm, out, lse, workspace,
-                       workspace_bytes, static_cast<cudaStream_t>(stream), &launches);
+                       workspace_bytes, static_cast<cudaStream_t>(stream), &launches, q_by_value);
     if (st == SPARK_OK) g_last_launches = launches;
     return st;
+}
+
+spark_status spark_decode_attn(const spark_params* p, const void* q, const void* pages,
+                               const int32_t* block_table, int32_t max_blocks,
+                               const int32_t* packed_lens, const float* qnorm, float* out, float* lse,
+                               void* workspace, size_t workspace_bytes, spark_stream_t stream)
+{
+    return decode_attn(p, q, pages, block_table, max_blocks, packed_lens, qnorm, out, lse, workspace, workspace_bytes,
+                       stream, false);
 }
 
 spark_status spark_decode_attn_host(const spark_params* p, const void* q_host, void* q_dev, const void* pages,
@@ -245,16 +255,22 @@ spark_status spark_decode_attn_host(const spark_params* p, const void* q_host, v
     if (st != SPARK_OK) return st;
     if (!q_host || !out_host) return SPARK_ERR_NULL;
     if (p->flags & SPARK_FLAG_HOST_MAPPED) {
-        // the kernel addresses the page-locked host buffers itself: 8-24 KB cross the bus inside the step
+        // The kernel writes the result (posted stores) straight into the page-locked host buffers.  The query
+        // travels inside the launch when it is small enough (read here, during the call); otherwise the kernel
+        // reads it over the bus during the step.
+        const size_t q_bytes = static_cast<size_t>(p->batch) * p->n_q_heads * p->head_dim * 2;
+        const bool by_value = p->dtype == SPARK_BF16 && p->recovery == SPARK_RECOVER_DEGENERATE &&
+                              value_keep(p->keep_v) == kHeadDim && q_bytes <= query_by_value_limit();
         void *dq = nullptr, *dout = nullptr, *dlse = nullptr;
-        if (cudaHostGetDevicePointer(&dq, const_cast<void*>(q_host), 0) != cudaSuccess ||
+        if ((!by_value && cudaHostGetDevicePointer(&dq, const_cast<void*>(q_host), 0) != cudaSuccess) ||
             cudaHostGetDevicePointer(&dout, out_host, 0) != cudaSuccess ||
             (lse_host && cudaHostGetDevicePointer(&dlse, lse_host, 0) != cudaSuccess)) {
             cudaGetLastError();                            // clear the sticky-free error of the failed lookup
             return SPARK_ERR_BAD_SHAPE;
         }
-        return spark_decode_attn(p, dq, pages, block_table, max_blocks, packed_lens, qnorm, static_cast<float*>(dout),
-                                 static_cast<float*>(dlse), workspace, workspace_bytes, stream);
+        return decode_attn(p, by_value ? q_host : dq, pages, block_table, max_blocks, packed_lens, qnorm,
+                           static_cast<float*>(dout), static_cast<float*>(dlse), workspace, workspace_bytes, stream,
+                           by_value);
     }
     if (!q_dev || !out_dev) return SPARK_ERR_NULL;
     if ((lse_dev == nullptr) != (lse_host == nullptr)) return SPARK_ERR_NULL;

@@ -142,7 +142,10 @@ int group_keep(int head_dim, int n_groups, const float* prune);
 spark_status launch_decode(const spark_params& p, const void* q, const void* pages,
                            const int32_t* block_table, int32_t max_blocks, const int32_t* packed_lens,
                            const float* qnorm, float* out, float* lse, void* workspace,
-                           size_t workspace_bytes, cudaStream_t stream, int* launches);
+                           size_t workspace_bytes, cudaStream_t stream, int* launches, bool q_by_value = false);
+// q_by_value: q is a HOST pointer and its bytes travel as a launch parameter (bf16 storage, degenerate recovery,
+// dense value rows, at most query_by_value_limit() bytes; anything else is refused)
+size_t query_by_value_limit();
 
 spark_status launch_append(const spark_params& p, const void* k_new, const void* v_new, void* pages,
                            const int32_t* block_table, int32_t max_blocks, const float* qnorm,

@@ -391,10 +391,12 @@ spark_status launch_decode_bf16_sampled(int G, const DecodeArgs& A, int dev, con
                                                   : launch_scalar_g<__nv_bfloat16, 2>(G, A, dev, info, stream);
 }
 
+size_t query_by_value_limit() { return kMaxQueryByValueBytes; }
+
 spark_status launch_decode(const spark_params& p, const void* q, const void* pages,
                            const int32_t* block_table, int32_t max_blocks, const int32_t* packed_lens,
                            const float* qnorm, float* out, float* lse, void* workspace,
-                           size_t workspace_bytes, cudaStream_t stream, int* launches)
+                           size_t workspace_bytes, cudaStream_t stream, int* launches, bool q_by_value)
 {
     (void)workspace_bytes;
     int dev = 0;
@@ -416,7 +418,9 @@ spark_status launch_decode(const spark_params& p, const void* q, const void* pag
     A.nslots = 0; A.slot_stride = 0; A.pps = 1; A.prefix_off = 0; A.ring_off = 0;
     A.overlap = (p.flags & SPARK_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
     A.seed = p.seed;
+    A.q_by_value = q_by_value ? 1 : 0;
     A.page_rows = A.L.ragged ? reinterpret_cast<const int*>(A.pages + rows_offset(p.n_pool_pages, A.L.page_bytes)) : nullptr;
+    if (q_by_value && (p.dtype != SPARK_BF16 || p.recovery != SPARK_RECOVER_DEGENERATE)) return SPARK_ERR_UNSUPPORTED;
     const spark_status st = (p.dtype != SPARK_BF16) ? launch_decode_f32(G, A, dev, info, stream)
                             : (p.recovery != SPARK_RECOVER_DEGENERATE) ? launch_decode_bf16_sampled(G, A, dev, info, stream)
                                                                        : launch_decode_bf16(G, A, dev, info, stream);

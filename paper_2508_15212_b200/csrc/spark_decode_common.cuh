@@ -45,7 +45,11 @@ struct DecodeArgs {
     int overlap;                             // launched as a programmatic dependent of the preceding kernel
     unsigned seed;                           // sampled recovery: seed of the per-entry draws
     const int* page_rows;                    // ragged pages: slot rows in use per pool page (else null: whole pages)
+    int q_by_value;                          // host side only: q is a HOST pointer whose bytes travel as a launch parameter
 };
+
+// largest query (bytes) that may travel as a launch parameter (kernel parameters are limited to 32764 bytes)
+constexpr int kMaxQueryByValueBytes = 24 * 1024;
 
 // control block at the start of dynamic shared memory
 constexpr int kCtrlBytes = 1024;                                 // full[32], empty[32], flags, plan
@@ -164,9 +168,9 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Launch helper: ordinary launch, or with the programmatic-stream-serialization attribute.
-template <typename Kernel>
+template <typename Kernel, typename... More>
 inline cudaError_t launch_decode_kernel(Kernel kernel, int grid, int threads, size_t smem, cudaStream_t stream,
-                                        const DecodeArgs& A)
+                                        const DecodeArgs& A, const More&... more)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -178,7 +182,7 @@ inline cudaError_t launch_decode_kernel(Kernel kernel, int grid, int threads, si
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = A.overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, A);
+    return cudaLaunchKernelEx(&cfg, kernel, A, more...);
 }
 
 template <int NT> __device__ __forceinline__ void consumer_sync()

@@ -24,6 +24,8 @@
 // a second mask instead of dense value rows; the warp first expands them (same nibble walk, zeros where
 // pruned) into a 4 KB tile of its own in shared memory, in the chunk-swizzled row layout of a dense
 // page, and the third contraction reads that tile.
+#include <cstring>
+
 #include "spark_decode_common.cuh"
 
 namespace spark {
@@ -217,8 +219,10 @@ __device__ __forceinline__ void sts_u32x4(unsigned addr, unsigned a, unsigned b,
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// The whole step; `q_src` is where the query rows are read from (global memory, or the launch's own
+// parameter block when the query travels with the launch).
 template <int G, bool kPV>
-__global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeArgs A)
+__device__ __forceinline__ void decode_bf16_body(const DecodeArgs& A, const void* q_src)
 {
     using S = SmemBf16<G, kPV>;
     constexpr bool kShared8 = (G <= 4);        // q' high and low parts share one 8-column operand
@@ -261,7 +265,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
         // ---- per-unit tables, built once per CTA: warp `hd` prepares query head hd ----
         if (warp < G) {
             const uint2 qr = *reinterpret_cast<const uint2*>(
-                static_cast<const unsigned short*>(A.q) +
+                static_cast<const unsigned short*>(q_src) +
                 (static_cast<int64_t>(b) * A.Hq + h * G + warp) * kHeadDim + 4 * lane);
             const float4 a4 = *reinterpret_cast<const float4*>(
                 A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + 4 * lane);
@@ -485,6 +489,37 @@ __global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeAr
 }
 
 template <int G, bool kPV>
+__global__ void __launch_bounds__(kThreads, 1) decode_bf16_kernel(const DecodeArgs A)
+{
+    decode_bf16_body<G, kPV>(A, A.q);
+}
+
+// The query as a kernel parameter: the launch itself carries the bytes to the GPU (no copy before the step,
+// no reads over the bus inside it).  Two sizes, so that a small query does not pay for a large parameter block.
+template <int kBytes> struct QueryBlob { uint4 v[kBytes / 16]; };
+constexpr int kBlobSmall = 8 * 1024, kBlobLarge = 24 * 1024;
+static_assert(kBlobLarge == kMaxQueryByValueBytes, "the launcher's limit is the large blob");
+
+template <int G, int kBytes>
+__global__ void __launch_bounds__(kThreads, 1) decode_bf16_qv_kernel(const __grid_constant__ DecodeArgs A,
+                                                                     const __grid_constant__ QueryBlob<kBytes> Q)
+{
+    decode_bf16_body<G, false>(A, &Q);
+}
+
+template <int G, int kBytes>
+static spark_status launch_bf16_qv(const DecodeArgs& A, int dev, int smem_optin, int grid, size_t smem, size_t q_bytes,
+                                   cudaStream_t stream)
+{
+    static unsigned char smem_raised[kMaxDevices] = {};
+    if (!allow_max_smem(decode_bf16_qv_kernel<G, kBytes>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
+    QueryBlob<kBytes> blob;                                 // A.q is a host pointer here; the bytes are taken now
+    memcpy(&blob, A.q, q_bytes);
+    return launch_decode_kernel(decode_bf16_qv_kernel<G, kBytes>, grid, kThreads, smem, stream, A, blob) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+template <int G, bool kPV>
 static spark_status launch_bf16(const DecodeArgs& A0, int dev, const DeviceInfo& info, cudaStream_t stream)
 {
     static unsigned char smem_raised[kMaxDevices] = {};
@@ -500,8 +535,15 @@ static spark_status launch_bf16(const DecodeArgs& A0, int dev, const DeviceInfo&
     if (ns < 2) return SPARK_ERR_UNSUPPORTED;
     A.nslots = ns;
     const size_t smem = A.ring_off + static_cast<size_t>(ns) * A.slot_stride;
-    if (!allow_max_smem(decode_bf16_kernel<G, kPV>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     const int grid = n_sms < kMaxCtas ? n_sms : kMaxCtas;
+    if (A.q_by_value) {
+        const size_t q_bytes = static_cast<size_t>(A.B) * A.Hq * kHeadDim * 2;
+        if (kPV || q_bytes > static_cast<size_t>(kBlobLarge)) return SPARK_ERR_UNSUPPORTED;
+        if (q_bytes <= static_cast<size_t>(kBlobSmall))
+            return launch_bf16_qv<G, kBlobSmall>(A, dev, smem_optin, grid, smem, q_bytes, stream);
+        return launch_bf16_qv<G, kBlobLarge>(A, dev, smem_optin, grid, smem, q_bytes, stream);
+    }
+    if (!allow_max_smem(decode_bf16_kernel<G, kPV>, dev, smem_optin, smem_raised)) return SPARK_ERR_CUDA;
     return launch_decode_kernel(decode_bf16_kernel<G, kPV>, grid, kThreads, smem, stream, A) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
 }

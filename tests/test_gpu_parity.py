@@ -454,6 +454,36 @@ def test_host_entry_point_staged_and_mapped_equal_the_device_call(dtype):
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("batch", [1, 3, 4])
+def test_host_mapped_query_travels_with_the_launch_when_it_fits(batch):
+    """SPARK_FLAG_HOST_MAPPED, bf16 storage: a query of up to 24 KB is read during the call and rides in the
+    launch (8 KB and 24 KB parameter blocks: batch 1 and 3 at 32 heads), so q_host may be overwritten as soon as
+    the call returns; a larger one (batch 4) is read by the kernel in stream order.  Same bits as the device
+    call, which is checked against the oracle here."""
+    lens = [200, 64, 17, 333][:batch]
+    wl = make("bf16", batch, 32, 8, lens, 8, 64, seed=171 + batch, sigma=1.0)
+    cache = SparkCache(batch=batch, n_q_heads=32, n_kv_heads=8, window=8, keep=64, dtype="bf16", max_tokens=max(lens))
+    cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
+    ref = cache.decode(wl.q)
+    _, _, o_ref, _ = oracle_side(wl.to("cpu"), 64)
+    assert float(np.abs(ref.cpu().numpy() - o_ref).max()) <= TOL["bf16"]
+    q_host = wl.q.cpu().pin_memory()
+    out_host = torch.full((batch, 32, 128), float("nan"), dtype=torch.float32).pin_memory()
+    cache.params.flags = B.SPARK_FLAG_HOST_MAPPED
+    call = cache.bind_decode_host(q_host, out_host)
+    by_value = batch * 32 * 256 <= 24 * 1024
+    for _ in range(2):
+        call()
+        if by_value:
+            q_host.zero_()                                      # the bytes were taken during the call
+        torch.cuda.synchronize()
+        assert torch.equal(out_host, ref.cpu())
+        q_host.copy_(wl.q.cpu())
+        out_host.fill_(float("nan"))
+    cache.params.flags = 0
+    assert cache.status() == 0
+
+
 def test_merge_attn_handles_empty_sides():
     o = torch.randn(2, 4, 128, device="cuda")
     zero = torch.zeros_like(o)
