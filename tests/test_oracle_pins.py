@@ -382,6 +382,43 @@ def test_eviction_boundary_inside_a_run_of_equal_pooled_values():
         assert list(kept[0, 0]) == run[:extra] + list(range(P, S))
 
 
+def test_eviction_votes_in_closed_form_uniform_and_one_hot_attention():
+    """Two cases whose votes are known without computing a softmax.  (a) All keys equal: every causal softmax
+    is uniform, so vote[t] = G * sum_w 1 / (S - W + w + 1) for every prefix token, all pooled values tie and the
+    lower positions are kept.  (b) Keys that are huge multiples of orthogonal directions, each window query
+    aligned with one prefix key: attention is one-hot, so vote[t] = number of (head, window row) pairs that
+    point at t, pooled[t] = the largest count within three positions, and the kept set follows by hand."""
+    B, Hq, Hkv, W, D, S = 1, 2, 1, 3, 8, 20
+    P = S - W
+    rng = np.random.default_rng(21)
+    q_win = rng.standard_normal((B, Hq, W, D)).astype(np.float32)
+    k = np.broadcast_to(rng.standard_normal((1, 1, 1, D)).astype(np.float32), (B, Hkv, S, D)).copy()
+    kept, n, vote, pooled = oracle.evict(q_win, k, [S], budget=9, pool=7, want_votes=True)
+    uniform = Hq * sum(1.0 / (P + w + 1) for w in range(W))
+    assert np.allclose(vote[0, 0, :P], uniform, rtol=1e-12) and np.allclose(pooled[0, 0, :P], uniform, rtol=1e-12)
+    assert list(kept[0, 0]) == list(range(9 - W)) + list(range(P, S))
+    # (b) one-hot attention: window query (g, w) points at prefix token target[g][w]
+    target = [[2, 2, 11], [2, 11, 15]]                                # counts: token 2 -> 3, token 11 -> 2, token 15 -> 1
+    k = np.zeros((B, Hkv, S, D), dtype=np.float32)
+    q_win = np.zeros((B, Hq, W, D), dtype=np.float32)
+    for j, tkn in enumerate((2, 11, 15)):
+        k[0, 0, tkn, j] = 1.0
+    for g in range(Hq):
+        for w in range(W):
+            q_win[0, g, w, (2, 11, 15).index(target[g][w])] = 400.0   # logit 400 / sqrt(8) against 0: one-hot in double
+    kept, n, vote, pooled = oracle.evict(q_win, k, [S], budget=W + 9, pool=7, want_votes=True)
+    want_vote = np.zeros(P)
+    want_vote[2], want_vote[11], want_vote[15] = 3.0, 2.0, 1.0
+    assert np.allclose(vote[0, 0, :P], want_vote, atol=1e-12)
+    want_pooled = np.zeros(P)
+    want_pooled[0:6] = 3.0                                            # |t - 2| <= 3, clamped at 0
+    want_pooled[8:15] = 2.0                                           # |t - 11| <= 3
+    want_pooled[15:17] = 1.0                                          # |t - 15| <= 3 where 11 does not reach (t = 15, 16; P = 17)
+    assert np.allclose(pooled[0, 0, :P], want_pooled, atol=1e-12)
+    # nine prefix tokens: the six at 3.0, then the three lowest of the seven at 2.0
+    assert list(kept[0, 0]) == [0, 1, 2, 3, 4, 5, 8, 9, 10] + list(range(P, S))
+
+
 # ---------------------------------------------------------------- value-channel pruning (App. "Pruning Value Cache Channels")
 def test_value_pruning_hand_rows_and_ties():
     # |v| = (3, 1, 0.5, 4, 1, 0, 2, 4): the three largest are channels 3 and 7 (4, tie -> lower first) and 0 (3)
