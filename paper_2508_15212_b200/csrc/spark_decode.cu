@@ -6,10 +6,12 @@
 // With a[j] = max(|q-bar_j|, eps) the reconstructed key is K~[t][j] = K[t][j] on kept channels and
 // mu[t] / a[j] on pruned ones, so for one query head
 //     q . K~[t] = sum_{j kept} q[j] * (K[t][j] - mu[t] / a[j])  +  mu[t] * sum_j q[j] / a[j].
-// This kernel evaluates that form with fp32 FMAs: a lane owns a token for the scores (it walks the set
+// This kernel evaluates that form on the CUDA cores: a lane owns a token for the scores (it walks the set
 // bits of the token's mask and gathers the query entries from a shared table) and four channels for
-// P.V.  fp32 caches are the small high-precision configuration; the bf16 tensor-core kernel carries the
-// bandwidth-bound workloads.
+// P.V.  fp32 caches are the small high-precision configuration (the bf16 tensor-core kernel carries the
+// bandwidth-bound workloads), so with the degenerate rule the table and the score sums are double: a
+// score then carries one rounding (to fp32, before the exponential) instead of the ~1e-6 relative error
+// of an fp32 sum over up to 128 cancelling terms, which at large logits was most of the output error.
 //
 // Sampled recovery (template parameter R = 1 Gaussian, 2 Exponential): every pruned entry of a token is a
 // draw w~ from the distribution built on the token's all-channel statistics (mean, population deviation;
@@ -19,6 +21,8 @@
 // the cache lives.  The algebraic folding of the degenerate rule does not apply: the lane walks all 128
 // channels of its token, which makes this the method's slow variant (the paper's ablation also ranks it
 // below the degenerate rule).
+#include <type_traits>
+
 #include "spark_decode_common.cuh"
 
 namespace spark {
@@ -54,10 +58,11 @@ template <> __device__ __forceinline__ float load_query<__nv_bfloat16>(const voi
 
 template <int G> struct SmemF32 {
     static constexpr int GP = ((G + 1 + 3) / 4) * 4;     // floats per table entry: G scaled queries + 1/a
+    static constexpr int GPD = ((G + 1 + 1) / 2) * 2;    // doubles per table entry (degenerate rule: double table)
     static constexpr int GPP = ((G + 3) / 4) * 4;        // floats per probability entry
     static constexpr int kQtab = kCtrlBytes;
-    static constexpr int kQsum = kQtab + kHeadDim * GP * 4;
-    static constexpr int kPscr = kQsum + 32;
+    static constexpr int kQsum = kQtab + kHeadDim * GPD * 8;     // sized for the double table (>= the float one)
+    static constexpr int kPscr = kQsum + 64;             // Qsum: [8] double
     static constexpr int kMerge = kPscr + kConsumerWarps * 32 * GPP * 4;
     static constexpr int kFixed = (kMerge + merge_bytes(kConsumerWarps, G) + 127) / 128 * 128;   // prefix and ring start here
 };
@@ -68,11 +73,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
     constexpr bool kBf16 = (sizeof(E) == 2);
     static_assert(!(kBf16 && R == 0), "bf16 storage with the degenerate rule runs on the tensor-core kernel");
     using S = SmemF32<G>;
-    constexpr int GP = S::GP, GPP = S::GPP;
+    // table element: double with the degenerate rule (fp32 storage, the high-precision configuration), else float
+    constexpr bool kDbl = (R == 0);
+    using TabT = typename std::conditional<kDbl, double, float>::type;
+    constexpr int GP = kDbl ? S::GPD : S::GP, GPP = S::GPP;
     extern __shared__ __align__(128) unsigned char smem[];
     const Ctrl C = make_ctrl(smem, A.prefix_off);
-    float* qtab = reinterpret_cast<float*>(smem + S::kQtab);
-    float* qsum = reinterpret_cast<float*>(smem + S::kQsum);
+    TabT* qtab = reinterpret_cast<TabT*>(smem + S::kQtab);
+    double* qsum = reinterpret_cast<double*>(smem + S::kQsum);
     float* pscr_all = reinterpret_cast<float*>(smem + S::kPscr);
     float* merge = reinterpret_cast<float*>(smem + S::kMerge);
     unsigned char* ring = smem + A.ring_off;
@@ -108,11 +116,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
         // ---- per-unit table: entry j = { q_0[j]*c, ..., q_{G-1}[j]*c, 1/a[j] },  c = scale*log2(e)
         for (int idx = tid; idx < kHeadDim * GP; idx += kConsumerThreads) {
             const int j = idx / GP, e = idx - j * GP;
-            float val = 0.f;
+            TabT val = 0;
             if (e < G)
-                val = load_query<E>(A.q, (static_cast<int64_t>(b) * A.Hq + h * G + e) * kHeadDim + j) * A.scale_log2e;
+                val = static_cast<TabT>(load_query<E>(A.q, (static_cast<int64_t>(b) * A.Hq + h * G + e) * kHeadDim + j)) *
+                      static_cast<TabT>(A.scale_log2e);
             else if (e == G)
-                val = 1.0f / A.qnorm[(static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + j];
+                val = static_cast<TabT>(1) / static_cast<TabT>(A.qnorm[(static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + j]);
             qtab[idx] = val;
         }
         consumer_sync<kConsumerThreads>();
@@ -120,12 +129,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
             double part = 0.0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const float* e = qtab + (lane * 4 + i) * GP;
+                const TabT* e = qtab + (lane * 4 + i) * GP;
                 part += static_cast<double>(e[warp]) * static_cast<double>(e[G]);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(kFull, part, o);
-            if (lane == 0) qsum[warp] = static_cast<float>(part);
+            if (lane == 0) qsum[warp] = part;
         }
         consumer_sync<kConsumerThreads>();
 
@@ -162,31 +171,37 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
                     float a[G];
 #pragma unroll
                     for (int gg = 0; gg < G; ++gg) a[gg] = 0.f;
-                    if (R == 0) {
-                        const float mu = *reinterpret_cast<const float*>(page + L.mu_off + p * 4);
+                    if constexpr (R == 0) {
+                        // fp32 storage is the high-precision configuration: the score of a token is summed in
+                        // double from a double table (products of two fp32 numbers are exact there), so that the
+                        // error of the step is that of the exponentials and of the fp32 value sums alone
+                        const double mu_d = static_cast<double>(*reinterpret_cast<const float*>(page + L.mu_off + p * 4));
+                        double ad[G];
+#pragma unroll
+                        for (int gg = 0; gg < G; ++gg) ad[gg] = 0.0;
 #pragma unroll
                         for (int wi = 0; wi < 4; ++wi) {
                             unsigned w = words[wi];
-                            const float* tb = qtab + wi * 32 * GP;
+                            const double* tb = qtab + wi * 32 * GP;
                             while (w) {
                                 const int bp = __ffs(w) - 1;
                                 w &= w - 1;
-                                const float* e = tb + bp * GP;
+                                const double* e = tb + bp * GP;
                                 const float kv = *reinterpret_cast<const float*>(vp);
                                 vp += kRowBytes;
-                                float tv[GP];
+                                double tv[GP];
 #pragma unroll
-                                for (int c4 = 0; c4 < GP / 4; ++c4) {
-                                    const float4 f = reinterpret_cast<const float4*>(e)[c4];
-                                    tv[4 * c4] = f.x; tv[4 * c4 + 1] = f.y; tv[4 * c4 + 2] = f.z; tv[4 * c4 + 3] = f.w;
+                                for (int c2 = 0; c2 < GP / 2; ++c2) {
+                                    const double2 f = reinterpret_cast<const double2*>(e)[c2];
+                                    tv[2 * c2] = f.x; tv[2 * c2 + 1] = f.y;
                                 }
-                                const float x = fmaf(-mu, tv[G], kv);
+                                const double x = fma(-mu_d, tv[G], static_cast<double>(kv));
 #pragma unroll
-                                for (int gg = 0; gg < G; ++gg) a[gg] = fmaf(tv[gg], x, a[gg]);
+                                for (int gg = 0; gg < G; ++gg) ad[gg] = fma(tv[gg], x, ad[gg]);
                             }
                         }
 #pragma unroll
-                        for (int gg = 0; gg < G; ++gg) s[gg] = fmaf(mu, qsum[gg], a[gg]);
+                        for (int gg = 0; gg < G; ++gg) s[gg] = static_cast<float>(fma(mu_d, qsum[gg], ad[gg]));
                     } else {
                         // sampled recovery: every channel contributes, kept ones their stored value, pruned
                         // ones a draw divided by a[j]
