@@ -271,17 +271,22 @@ def oracle_on_kept_tokens(wl_cpu, kept, n, keep):
                                                    ("bf16", [2000], 32, 256, 7),
                                                    ("f32", [500, 64], 16, 96, 2)])
 def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
+    check_eviction_case(dtype, lens, W, budget, G)
+
+
+def check_eviction_case(dtype, lens, W, budget, G, keep=64, Hkv=2, pool=7, seed=None):
     """Three checks, none of them conditional on the other: (1) the evicted token sets against the oracle's
     (exact where the pooled votes at the budget boundary are not a near-tie); (2) pruning and decode of the
     evicting call against the oracle run on the SAME token set (the one the GPU kept); (3) pruning and decode
     of the oracle's token set, gathered and fed to both sides through the non-evicting call.  A near-tie in
     (1) can therefore never hide a pruning or decode error."""
-    keep, Hkv, Bn = 64, 2, len(lens)
-    wl = make(dtype, Bn, Hkv * G, Hkv, lens, W, keep, seed=130 + G, sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
+    Bn = len(lens)
+    wl = make(dtype, Bn, Hkv * G, Hkv, lens, W, keep, seed=130 + G if seed is None else seed,
+              sigma=1.0 if dtype == "bf16" else 0.5, gap=False)
     wl_cpu = wl.to("cpu")
-    kept_ref, n_ref, gaps = oracle_evicted_sets(wl_cpu, budget, 7)
+    kept_ref, n_ref, gaps = oracle_evicted_sets(wl_cpu, budget, pool)
     cache = SparkCache(batch=Bn, n_q_heads=Hkv * G, n_kv_heads=Hkv, window=W, keep=keep, dtype=dtype,
-                       max_tokens=max(lens), token_budget=budget, pool_kernel=7, guard=True)
+                       max_tokens=max(lens), token_budget=budget, pool_kernel=pool, guard=True)
     cache.compress(wl.q_win, wl.k, wl.v, wl.seq_lens)
     assert cache.status() == 0
     assert cache.packed_lens.cpu().tolist() == n_ref.tolist()
@@ -290,7 +295,9 @@ def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
     for b in range(Bn):
         for h in range(Hkv):
             a_, r_ = kept[b, h, :n_ref[b]], kept_ref[b, h, :n_ref[b]]
-            assert (np.diff(a_) > 0).all() and a_[-W:].tolist() == list(range(lens[b] - W, lens[b]))
+            assert (np.diff(a_) > 0).all()
+            if lens[b] >= W:
+                assert a_[-W:].tolist() == list(range(lens[b] - W, lens[b]))
             if gaps[b, h] > 1e-4:
                 assert np.array_equal(a_, r_), f"evicted set differs at unit ({b},{h}), gap {gaps[b, h]:.2e}"
             else:
@@ -298,8 +305,10 @@ def test_eviction_then_pruning_against_oracle(dtype, lens, W, budget, G):
     # (2) the evicting call's pages and output against the oracle on the GPU's own token set
     c_gpu, out_gpu_ref, _, _ = oracle_on_kept_tokens(wl_cpu, kept, n_ref, keep)
     u = cache.unpack(want_vals=False, want_v=False)
-    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c_gpu["mask"])
-    assert np.allclose(u["mu"].cpu().numpy(), c_gpu["mu"], rtol=1e-6, atol=0)
+    m = min(max(lens), budget)                              # tokens a unit can hold: the unpacked and the oracle arrays
+    assert int(n_ref.max()) <= m                            # are sized max(lens) and budget
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32)[:, :, :m], c_gpu["mask"][:, :, :m])
+    assert np.allclose(u["mu"].cpu().numpy()[:, :, :m], c_gpu["mu"][:, :, :m], rtol=1e-6, atol=0)
     out = cache.decode(wl.q)
     assert cache.status() == 0
     d = float(np.abs(out.cpu().numpy() - out_gpu_ref).max())

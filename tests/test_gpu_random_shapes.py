@@ -11,7 +11,7 @@ import random
 import pytest
 import torch
 
-from test_gpu_parity import built, check_case, make                      # noqa: F401  (fixture + helpers)
+from test_gpu_parity import built, check_case, check_eviction_case, make  # noqa: F401  (fixture + helpers)
 from workloads.batches import permuted_block_table
 
 pytestmark = pytest.mark.gpu
@@ -56,3 +56,83 @@ def test_random_shape(seed):
         table, n_pages = permuted_block_table(c["Bn"], c["Hkv"], c["lens"], "cuda", seed=seed)
         n_pool = n_pages + 3                            # spare pages that nothing may touch
     check_case(wl, c["keep"], block_table=table, n_pool_pages=n_pool, keep_v=c["keep_v"])
+
+
+def draw_eviction_case(seed):
+    rnd = random.Random(seed)
+    dtype = rnd.choice(["bf16", "bf16", "f32"])
+    W = rnd.choice([4, 8, 16, 32, 64])
+    G = rnd.choice([1, 2, 4, 4, 7, 8])                  # G * W above 256 leaves the tensor-core votes for the fallback
+    Hkv = rnd.choice([1, 2, 3])
+    budget = W + rnd.choice([1, 5, 30, 64, 200, 448])
+    pool = rnd.choice([1, 3, 7, 7, 7])
+    keep = rnd.choice([25, 64, 64, 100])
+    Bn = rnd.choice([1, 2, 4])
+    lens = []
+    for _ in range(Bn):
+        kind = rnd.random()
+        if kind < 0.2:
+            n = rnd.randint(max(1, W // 2), budget)                        # nothing to evict (at or under the budget)
+        elif kind < 0.35:
+            n = budget + rnd.randint(1, 3)                                 # evicts one to three tokens
+        else:
+            n = rnd.randint(budget + 1, budget + rnd.choice([50, 700, 3000]))
+        lens.append(n)
+    return dict(dtype=dtype, lens=lens, W=W, budget=budget, G=G, keep=keep, Hkv=Hkv, pool=pool)
+
+
+@pytest.mark.parametrize("seed", list(range(500, 540)))
+def test_random_eviction_shape(seed):
+    c = draw_eviction_case(seed)
+    check_eviction_case(c["dtype"], c["lens"], c["W"], c["budget"], c["G"], keep=c["keep"], Hkv=c["Hkv"],
+                        pool=c["pool"], seed=seed)
+
+
+@pytest.mark.parametrize("seed", list(range(700, 724)))
+def test_random_append_mix(seed):
+    """Prefill a random ragged batch, then grow it by a random mix of one-token appends and block appends (in a
+    paged pool or a contiguous cache, with or without value pruning): the cache must equal the oracle's pruning of
+    the full sequences with the prefill window statistics, and the decode output must match."""
+    import numpy as np
+    from test_gpu_parity import TOL, oracle_side
+    from paper_2508_15212_b200.cache import SparkCache
+    rnd = random.Random(seed)
+    dtype = rnd.choice(["bf16", "bf16", "f32"])
+    G, Hkv, Bn = rnd.choice([1, 2, 4, 7]), rnd.choice([1, 2, 3]), rnd.choice([1, 2, 4])
+    keep = rnd.choice([25, 38, 64, 127, 128])
+    keep_v = rnd.choice([0, 0, 64])
+    lens0 = [rnd.choice([0, 1, 15, 16, 17, rnd.randint(1, 300)]) for _ in range(Bn)]
+    n_app = rnd.randint(1, 70)
+    lens1 = [l + n_app for l in lens0]
+    S = max(lens1)
+    full = make(dtype, Bn, G * Hkv, Hkv, lens1, 8, keep, seed=seed, sigma=1.0 if dtype == "bf16" else 0.5)
+    table, n_pool = None, None
+    if rnd.random() < 0.5:
+        table, n_pages = permuted_block_table(Bn, Hkv, lens1, "cuda", seed=seed)
+        n_pool = n_pages + 2
+    cache = SparkCache(batch=Bn, n_q_heads=G * Hkv, n_kv_heads=Hkv, window=8, keep=keep, dtype=dtype, max_tokens=S,
+                       block_table=table, n_pool_pages=n_pool, keep_v=keep_v, guard=True)
+    lens0_t = torch.tensor(lens0, dtype=torch.int32, device="cuda")
+    cache.compress(full.q_win, full.k, full.v, lens0_t)
+    done = 0
+    while done < n_app:
+        n = min(n_app - done, rnd.choice([1, 1, 2, 5, 16, 33]))
+        idx = (lens0_t.long().view(Bn, 1, 1, 1) + done + torch.arange(n, device="cuda").view(1, 1, n, 1))
+        idx = idx.expand(Bn, Hkv, n, 128)
+        k_blk, v_blk = full.k.gather(2, idx).contiguous(), full.v.gather(2, idx).contiguous()
+        if n == 1 and rnd.random() < 0.7:
+            cache.append(k_blk[:, :, 0].contiguous(), v_blk[:, :, 0].contiguous())
+        else:
+            cache.append_block(k_blk, v_blk)
+        done += n
+    assert cache.status() == 0 and cache.broken_guards() == []
+    assert cache.packed_lens.cpu().tolist() == lens1
+    a, c, o_ref, _ = oracle_side(full.to("cpu"), keep, keep_v)
+    u = cache.unpack(want_vmask=True)
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c["mask"])
+    assert np.allclose(u["mu"].cpu().numpy(), c["mu"], rtol=1e-6, atol=0)
+    if c["vmask"] is not None:
+        assert np.array_equal(u["vmask"].cpu().numpy().view(np.uint32), c["vmask"])
+    out = cache.decode(full.q)
+    assert cache.status() == 0 and cache.broken_guards() == []
+    assert float(np.abs(out.cpu().numpy() - o_ref).max()) <= TOL[dtype]
