@@ -136,3 +136,35 @@ def test_random_append_mix(seed):
     out = cache.decode(full.q)
     assert cache.status() == 0 and cache.broken_guards() == []
     assert float(np.abs(out.cpu().numpy() - o_ref).max()) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("seed", list(range(800, 830)))
+def test_random_variant_shape(seed):
+    """The ratio-free selection rules (Sec. "Ablation Studies", adaptive variants) and the sampled recovery
+    distributions (Sec. "Channel Recovery") on random ragged batches, paged or contiguous."""
+    import test_gpu_variants as V
+    from paper_2508_15212_b200 import binding as B
+    rnd = random.Random(seed)
+    dtype = rnd.choice(["bf16", "bf16", "f32"])
+    G, Hkv, Bn = rnd.choice([1, 2, 4, 5, 7, 8]), rnd.choice([1, 2, 3]), rnd.choice([1, 2, 3, 6])
+    cap_len = rnd.choice([40, 200, 900])
+    lens = [rnd.choice([0, 16, 17, rnd.randint(1, cap_len)]) for _ in range(Bn)]
+    if max(lens) == 0:
+        lens[0] = cap_len
+    wl = V.make(dtype, Bn, G * Hkv, Hkv, lens, rnd.choice([4, 8, 32]), seed)
+    table, n_pool = None, None
+    if rnd.random() < 0.4:
+        table, n_pages = permuted_block_table(Bn, Hkv, lens, "cuda", seed=seed)
+        n_pool = n_pages + 2
+    kind = rnd.choice(["top_p", "groups", "gaussian", "exponential", "sampled_top_p"])
+    if kind == "top_p":
+        V.check_selection(wl, rnd.choice([128, 96, 40]), top_p=rnd.choice([0.5, 0.9, 0.99, 0.999]),
+                          block_table=table, n_pool_pages=n_pool)
+    elif kind == "groups":
+        ratios = rnd.choice([[0.25, 0.5, 0.75, 1.0], [0.1, 0.3, 0.5, 0.7, 0.9], [0.0, 1.0], [0.5], [0.2, 0.4, 0.6]])
+        V.check_selection(wl, B.spark_group_keep(128, ratios), group_prune=ratios, block_table=table, n_pool_pages=n_pool)
+    elif kind == "sampled_top_p":
+        V.check_sampled(wl, 128, rnd.choice([1, 2]), seed, top_p=0.95, block_table=table, n_pool_pages=n_pool)
+    else:
+        V.check_sampled(wl, rnd.choice([25, 64, 100]), 1 if kind == "gaussian" else 2, seed,
+                        block_table=table, n_pool_pages=n_pool)
