@@ -27,20 +27,20 @@ window_qnorm_kernel(const void* __restrict__ q_win, int Hq, int Hkv, int W, floa
 {
     const int h = blockIdx.x, b = blockIdx.y, j = threadIdx.x;
     const int G = Hq / Hkv;
+    // the group's G*W window rows are consecutive in memory, (g outer, w inner)
+    const int64_t base = ((static_cast<int64_t>(b) * Hq + h * G) * W) * kHeadDim + j;
+    const int rows = G * W;
     double acc = 0.0;
-    for (int g = 0; g < G; ++g) {
-        const int64_t base = ((static_cast<int64_t>(b) * Hq + (h * G + g)) * W) * kHeadDim + j;
-        int w = 0;
-        for (; w + 8 <= W; w += 8) {                       // eight loads in flight, summed in order
-            float x[8];
+    int r = 0;
+    for (; r + 32 <= rows; r += 32) {                      // thirty-two loads in flight, summed in order
+        float x[32];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) x[u] = Elem<E>::load(q_win, base + static_cast<int64_t>(w + u) * kHeadDim);
+        for (int u = 0; u < 32; ++u) x[u] = Elem<E>::load(q_win, base + static_cast<int64_t>(r + u) * kHeadDim);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc += static_cast<double>(x[u]);
-        }
-        for (; w < W; ++w)
-            acc += static_cast<double>(Elem<E>::load(q_win, base + static_cast<int64_t>(w) * kHeadDim));
+        for (int u = 0; u < 32; ++u) acc += static_cast<double>(x[u]);
     }
+    for (; r < rows; ++r)
+        acc += static_cast<double>(Elem<E>::load(q_win, base + static_cast<int64_t>(r) * kHeadDim));
     const float m = static_cast<float>(acc / static_cast<double>(G * W));
     qnorm[(static_cast<int64_t>(b) * Hkv + h) * kHeadDim + j] = fmaxf(fabsf(m), eps);
     if (packed_lens && h == 0 && j == 0) {
