@@ -34,19 +34,36 @@ constexpr int kStepTokens = 2 * kPageTokens;              // a lane per token: t
 
 // one sampled saliency: Gaussian N(mu, sigma^2) by Box-Muller (R = 1) or Exponential with mean mu by
 // inversion (R = 2), from the counter (unit, t, j)
-template <int R>
-__device__ __forceinline__ float sample_saliency(unsigned seed, unsigned long long unit_t, int j, float mu, float sigma)
+// the 64 mixed bits of the counter (unit, t, j)
+__device__ __forceinline__ unsigned long long draw_bits(unsigned seed, unsigned long long unit_t, int j)
 {
     unsigned long long z = unit_t ^ static_cast<unsigned long long>(j);
     z += static_cast<unsigned long long>(seed) * 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
     z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-    z ^= z >> 31;
+    return z ^ (z >> 31);
+}
+
+template <int R>
+__device__ __forceinline__ float sample_saliency(unsigned seed, unsigned long long unit_t, int j, float mu, float sigma)
+{
+    const unsigned long long z = draw_bits(seed, unit_t, j);
     // (x + 0.5) / 2^24 with x < 2^24: the sum needs 25 bits, so it is formed in double and rounded once
     const float u1 = static_cast<float>((static_cast<double>(z >> 40) + 0.5) * (1.0 / 16777216.0));
     if (R == 2) return -mu * logf(u1);
     const float u2 = static_cast<float>((static_cast<double>((z >> 16) & 0xFFFFFFull) + 0.5) * (1.0 / 16777216.0));
     return fmaf(sigma * sqrtf(-2.0f * logf(u1)), cospif(2.0f * u2), mu);
+}
+
+// the same draw evaluated in double: fp32 storage, where the output is held to the fp32 bar
+template <int R>
+__device__ __forceinline__ double sample_saliency_f64(unsigned seed, unsigned long long unit_t, int j, float mu, float sigma)
+{
+    const unsigned long long z = draw_bits(seed, unit_t, j);
+    const double u1 = (static_cast<double>(z >> 40) + 0.5) * (1.0 / 16777216.0);
+    if (R == 2) return -static_cast<double>(mu) * log(u1);
+    const double u2 = (static_cast<double>((z >> 16) & 0xFFFFFFull) + 0.5) * (1.0 / 16777216.0);
+    return fma(static_cast<double>(sigma) * sqrt(-2.0 * log(u1)), cospi(2.0 * u2), static_cast<double>(mu));
 }
 
 template <typename E> __device__ __forceinline__ float load_query(const void* q, int64_t i);
@@ -168,9 +185,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
                     // element (p & 7) * 2 + (p >> 3); rows are 16 elements apart
                     const unsigned char* vp = page + L.vals_off + (kBf16 ? ((p & 7) * 2 + (p >> 3)) * 2 : p * 4);
                     constexpr int kRowBytes = kPageTokens * static_cast<int>(sizeof(E));
-                    float a[G];
+                    // sampled rules: fp32 storage sums the score in double as well (bf16 storage: fp32 is ample)
+                    using AccT = typename std::conditional<kBf16, float, double>::type;
+                    AccT a[G];
 #pragma unroll
-                    for (int gg = 0; gg < G; ++gg) a[gg] = 0.f;
+                    for (int gg = 0; gg < G; ++gg) a[gg] = 0;
                     if constexpr (R == 0) {
                         // fp32 storage is the high-precision configuration: the score of a token is summed in
                         // double from a double table (products of two fp32 numbers are exact there), so that the
@@ -223,20 +242,23 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_scalar_kernel(const 
                                     const float4 f = reinterpret_cast<const float4*>(e)[c4];
                                     tv[4 * c4] = f.x; tv[4 * c4 + 1] = f.y; tv[4 * c4 + 2] = f.z; tv[4 * c4 + 3] = f.w;
                                 }
-                                float x;
+                                AccT x;
                                 if ((w >> bp) & 1u) {
                                     x = kBf16 ? bf16_bits_to_float(*reinterpret_cast<const unsigned short*>(vp))
                                               : *reinterpret_cast<const float*>(vp);
                                     vp += kRowBytes;
-                                } else {
+                                } else if constexpr (kBf16) {
                                     x = sample_saliency<R>(A.seed, unit_t, j, mean, dev) * tv[G];
+                                } else {
+                                    x = sample_saliency_f64<R>(A.seed, unit_t, j, mean, dev) * static_cast<double>(tv[G]);
                                 }
 #pragma unroll
-                                for (int gg = 0; gg < G; ++gg) a[gg] = fmaf(tv[gg], x, a[gg]);
+                                for (int gg = 0; gg < G; ++gg)
+                                    a[gg] = fma(static_cast<AccT>(tv[gg]), x, a[gg]);
                             }
                         }
 #pragma unroll
-                        for (int gg = 0; gg < G; ++gg) s[gg] = a[gg];
+                        for (int gg = 0; gg < G; ++gg) s[gg] = static_cast<float>(a[gg]);
                     }
                 } else {
 #pragma unroll
