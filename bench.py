@@ -537,7 +537,7 @@ def main():
     e2e_us = dist_utils.max_over_ranks(e0.elapsed_time(e1), dist, "cuda") * 1e3 / e2e_steps
     # the same call with SPARK_FLAG_HOST_MAPPED: the query travels inside the launch (or is read by the kernel)
     # and the kernel writes the result into the pinned host buffer itself, no staging copies; reported beside
-    # the staged figure, which stays the e2e value
+    # the staged figure; the e2e value is the faster of the two
     for c in work.caches:
         c.params.flags = B.SPARK_FLAG_HOST_MAPPED
     for i in range(20):
@@ -608,10 +608,17 @@ def main():
             "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
             "algorithmic_bytes_per_step": work.alg_bytes,
             "clocks": t_plain["clocks"],
-            "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "value_host_mapped": e2e_mapped_us,
-                    "note": ("packed cache resident; per step one spark_decode_attn_host call (pinned q -> device, the "
-                             "decode step, out -> pinned host) and a stream synchronize")},
+            "e2e": {"value": min(e2e_us, e2e_mapped_us), "unit": "us/step", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "transport": ("SPARK_FLAG_HOST_MAPPED" if e2e_mapped_us < e2e_us else "staged copies"),
+                    "value_staged_copies": e2e_us, "value_host_mapped": e2e_mapped_us,
+                    "note": ("packed cache resident; per step one spark_decode_attn_host call (query in pinned host "
+                             "memory -> device, the decode step, result -> pinned host memory) and a stream "
+                             "synchronize; timed with both transports of that call, the value is the faster one: "
+                             "staged = cudaMemcpyAsync in, kernel, cudaMemcpyAsync out; SPARK_FLAG_HOST_MAPPED = the "
+                             "query bytes travel inside the kernel launch (up to 24 KB, else the kernel reads them "
+                             "from the host buffer) and the kernel writes the result into the host buffer; the same "
+                             "bytes cross the bus either way")},
             "gpu_launches": t_plain["launches"] * B.spark_last_launch_count(),
             "launches_per_step": lps,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
