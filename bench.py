@@ -14,8 +14,9 @@ Timing.  The steps are captured in CUDA graphs and timed with CUDA events on the
   value_pdl      the same K steps launched with SPARK_FLAG_OVERLAP_PREVIOUS (programmatic dependent launch:
                  step i+1 may start its page stream while step i drains), a pipelined-throughput figure that
                  holds only when the kernel enqueued before the step does not write the cache.
-With the default workload (the 32K headline configuration) the run also times the 4x128K and the evicted
-32x2048 configurations and reports them under "sweep" in the same JSON line (--no-sweep skips them).
+With the default workload (the 32K headline configuration) the run also times the 4x128K, the evicted
+32x2048 and the 28-layer Qwen-shape configurations and reports them under "sweep" in the same JSON line
+(--no-sweep skips them).
 
 With N > 1 (torchrun) every rank runs the same workload on its own GPU with no data-path collective (weak
 scaling); the reported time is the max over ranks.  --impl reference times the CPU oracle on the host cores
@@ -576,7 +577,7 @@ def main():
     sweep = []
     if world == 1 and args.config == 1 and not args.no_sweep and not keep_v and not args.batch and not args.keep \
             and variant is None:
-        for idx in (2, 3):
+        for idx in (2, 3, 4):
             torch.cuda.empty_cache()
             cfg_s, keep_s = resolve(idx)
             work_s = build_work(idx, cfg_s, keep_s, 0, rank, torch, B)
