@@ -653,7 +653,8 @@ __global__ void __launch_bounds__(128, 8) compress_pages4_kernel(CompressArgs A)
 // ------------------------------------------------------------------------------------------------
 // Decode-time append: one new token per sequence is pruned with the sequence's prefill statistics
 // (qnorm) and written into the next token slot of its last page (a fresh page is zeroed first).
-// One warp per (sequence, KV head); a second one-thread-per-sequence kernel advances packed_lens.
+// One warp per (sequence, KV head).  With more than 32 KV heads: a CTA per warp, and a second
+// one-thread-per-sequence kernel advances packed_lens; otherwise one launch does both (below).
 // ------------------------------------------------------------------------------------------------
 struct AppendArgs {
     const void* k_new;
@@ -701,6 +702,45 @@ __global__ void __launch_bounds__(32) append_token_kernel(AppendArgs A)
     const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
     const int n_kept = pack_token_kv<kBf16, kRank>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
     if (rows && lane == 0) atomicMax(rows, n_kept);
+}
+
+// The same for up to 32 KV heads in ONE launch: a CTA per sequence, a warp per KV head.  Every warp reads the
+// sequence's length before the first barrier and thread 0 advances it after the second, so no warp can see
+// the advanced length.
+template <typename E, bool kRank>
+__global__ void __launch_bounds__(1024) append_token_cta_kernel(AppendArgs A)
+{
+    constexpr bool kBf16 = (sizeof(E) == 2);
+    const int b = blockIdx.x, h = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const PageLayout L = A.L;
+    const int t = A.packed_lens[b];
+    __syncthreads();
+    const int blk = t / kPageTokens, p = t - blk * kPageTokens;
+    const bool room = t >= 0 && blk < A.max_blocks;
+    if (!room) {                                               // no room: recorded, nothing written
+        if (threadIdx.x == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+    } else {
+        const int64_t entry = (static_cast<int64_t>(b) * A.Hkv + h) * A.max_blocks + blk;
+        const int64_t page_id = A.block_table ? A.block_table[entry] : entry;
+        if (page_id < 0 || page_id >= A.n_pool_pages) {
+            if (lane == 0) record_error(A.status, SPARK_ERR_DEVICE_BOUNDS);
+        } else {
+            unsigned char* page = A.pages + page_id * L.page_bytes;
+            int* rows = L.ragged ? reinterpret_cast<int*>(A.pages + rows_offset(A.n_pool_pages, L.page_bytes)) + page_id : nullptr;
+            if (p == 0) {                                      // first token of a page: clear it
+                for (int i = lane; i < L.page_bytes / 16; i += 32) reinterpret_cast<uint4*>(page)[i] = make_uint4(0, 0, 0, 0);
+                if (rows && lane == 0) *rows = 0;
+                __syncwarp();
+            }
+            const float4 a4 = reinterpret_cast<const float4*>(A.qnorm + (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim)[lane];
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+            const int64_t row = (static_cast<int64_t>(b) * A.Hkv + h) * kHeadDim + lane * 4;
+            const int n_kept = pack_token_kv<kBf16, kRank>(page, L, p, lane, a, A.k_new, A.v_new, row, A.inv_pruned, A.sel);
+            if (rows && lane == 0) atomicMax(rows, n_kept);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && room) A.packed_lens[b] = t + 1;
 }
 
 __global__ void append_advance_kernel(AppendArgs A)
@@ -810,8 +850,20 @@ spark_status launch_append(const spark_params& p, const void* k_new, const void*
     A.inv_pruned = p.keep < kHeadDim ? 1.0 / static_cast<double>(kHeadDim - p.keep) : 0.0;
     A.sel = make_select(p);
     A.status = static_cast<int*>(workspace);
-    const dim3 grid(p.n_kv_heads, p.batch);
     const bool rank = p.select != SPARK_SELECT_FIXED;
+    if (p.n_kv_heads <= 32) {                                  // one launch: a CTA per sequence, a warp per KV head
+        const int threads = p.n_kv_heads * 32;
+        if (p.dtype == SPARK_BF16) {
+            if (rank) append_token_cta_kernel<__nv_bfloat16, true><<<p.batch, threads, 0, stream>>>(A);
+            else append_token_cta_kernel<__nv_bfloat16, false><<<p.batch, threads, 0, stream>>>(A);
+        } else {
+            if (rank) append_token_cta_kernel<float, true><<<p.batch, threads, 0, stream>>>(A);
+            else append_token_cta_kernel<float, false><<<p.batch, threads, 0, stream>>>(A);
+        }
+        *launches += 1;
+        return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    }
+    const dim3 grid(p.n_kv_heads, p.batch);
     if (p.dtype == SPARK_BF16) {
         if (rank) append_token_kernel<__nv_bfloat16, true><<<grid, 32, 0, stream>>>(A);
         else append_token_kernel<__nv_bfloat16, false><<<grid, 32, 0, stream>>>(A);

@@ -362,6 +362,7 @@ def test_append_tokens_equals_compressing_the_longer_sequence(dtype, keep):
     for i in range(n_app):
         idx = (lens0_t.long() + i).view(3, 1, 1, 1).expand(3, 2, 1, 128)
         cache.append(full.k.gather(2, idx).squeeze(2).contiguous(), full.v.gather(2, idx).squeeze(2).contiguous())
+        assert B.lib().spark_last_launch_count() == 1             # a CTA per sequence, a warp per KV head
     assert cache.status() == 0
     assert cache.packed_lens.cpu().tolist() == [l + n_app for l in lens0]
     wl_cpu = full.to("cpu")
@@ -377,6 +378,27 @@ def test_append_tokens_equals_compressing_the_longer_sequence(dtype, keep):
     small.compress(one.q_win, one.k, one.v, one.seq_lens)
     small.append(one.k[:, :, 0].contiguous(), one.v[:, :, 0].contiguous())
     assert small.packed_lens.cpu().tolist() == [16] and B.spark_read_status(small.ws_compress) == 6
+
+
+def test_append_with_more_than_32_kv_heads():
+    """Up to 32 KV heads a CTA per sequence appends all heads in one launch; beyond that the per-head launch plus
+    the length update is used.  Same result either way (oracle pruning of the longer sequence)."""
+    lens0, n_app, Hkv, keep = [20, 5], 14, 40, 64
+    full = make("bf16", 2, Hkv, Hkv, [l + n_app for l in lens0], 4, keep, seed=154)
+    S = max(lens0) + n_app
+    cache = SparkCache(batch=2, n_q_heads=Hkv, n_kv_heads=Hkv, window=4, keep=keep, dtype="bf16", max_tokens=S, guard=True)
+    lens0_t = torch.tensor(lens0, dtype=torch.int32, device="cuda")
+    cache.compress(full.q_win, full.k, full.v, lens0_t)
+    for i in range(n_app):
+        idx = (lens0_t.long() + i).view(2, 1, 1, 1).expand(2, Hkv, 1, 128)
+        cache.append(full.k.gather(2, idx).squeeze(2).contiguous(), full.v.gather(2, idx).squeeze(2).contiguous())
+        assert B.lib().spark_last_launch_count() == 2
+    assert cache.status() == 0 and cache.broken_guards() == []
+    assert cache.packed_lens.cpu().tolist() == [l + n_app for l in lens0]
+    a, c, o_ref, _ = oracle_side(full.to("cpu"), keep)
+    u = cache.unpack(want_vals=False, want_v=False)
+    assert np.array_equal(u["mask"].cpu().numpy().view(np.uint32), c["mask"])
+    assert float(np.abs(cache.decode(full.q).cpu().numpy() - o_ref).max()) <= TOL["bf16"]
 
 
 def test_block_append_equals_appending_one_token_at_a_time():
